@@ -1,0 +1,166 @@
+"""CLT-k oracle -- TEST INFRASTRUCTURE, never part of the product path.
+
+Thin ctypes marshalling around ``cltk_oracle.c`` (plain C, fp32 and fp64): a
+slow, single-threaded, step-by-step statement of one ScaleCom iteration
+(Algorithm 1; CLT-k compressor Eq. 2-3; low-pass-filtered memory Eq. 4).
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+import this package.  All arithmetic lives in the C file; this module only
+converts numpy arrays to pointers.
+
+Pins (see tests/test_oracle_pins.py): brute-force rank counting and subset
+enumeration on tiny d (Eq. 2), k = d reducing to dense averaged SGD
+(Algorithm 1 lines 10-12), n = 1 with beta = 1 reducing to classical
+error-feedback top-k (Remark 1), acc = sparse + residual (Eq. 4), leader
+cycling (Algorithm 1 line 6), commutativity (Eq. 1), the virtual-sequence
+identity of Appendix D.1, the contraction identity of Appendix C and a
+library top-k cross-check.  No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "cltk_oracle.c")
+_INC = os.path.join(_HERE, "cltk_oracle_body.inc")
+_LIB = os.path.join(_HERE, "libcltk_oracle.so")
+
+CFLAGS = ["-std=c99", "-O2", "-ffp-contract=off", "-fPIC", "-shared"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    stale = (not os.path.exists(_LIB)
+             or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_INC)))
+    if force or stale:
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.run(["gcc", *CFLAGS, _SRC, "-o", tmp], check=True, cwd=_HERE)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        i32, i64 = ctypes.c_int32, ctypes.c_int64
+        vp = ctypes.c_void_p
+        for sfx, real in (("f32", ctypes.c_float), ("f64", ctypes.c_double)):
+            f = getattr(_lib, "oracle_rank_" + sfx); f.restype = i64; f.argtypes = [vp, i64, i64]
+            f = getattr(_lib, "oracle_topk_" + sfx); f.restype = ctypes.c_int; f.argtypes = [vp, i64, i64, vp, vp]
+            f = getattr(_lib, "oracle_accumulate_" + sfx); f.restype = None; f.argtypes = [vp, vp, i64, vp]
+            f = getattr(_lib, "oracle_learner_" + sfx); f.restype = None
+            f.argtypes = [vp, vp, i64, vp, i64, vp, real, vp]
+            f = getattr(_lib, "oracle_reduce_" + sfx); f.restype = None; f.argtypes = [vp, i32, i64, vp]
+            f = getattr(_lib, "oracle_apply_" + sfx); f.restype = None; f.argtypes = [vp, vp, vp, i64, real]
+            f = getattr(_lib, "oracle_step_" + sfx); f.restype = ctypes.c_int
+            f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, vp, vp, vp]
+    return _lib
+
+
+def _sfx(dtype) -> str:
+    dtype = np.dtype(dtype)
+    if dtype == np.float32:
+        return "f32"
+    if dtype == np.float64:
+        return "f64"
+    raise TypeError("oracle works in float32 or float64, got %s" % dtype)
+
+
+def _chk(a: np.ndarray, dtype, shape=None) -> np.ndarray:
+    if not isinstance(a, np.ndarray) or a.dtype != np.dtype(dtype) or not a.flags.c_contiguous:
+        raise TypeError("expected a C-contiguous %s ndarray" % np.dtype(dtype))
+    if shape is not None and tuple(a.shape) != tuple(shape):
+        raise ValueError("expected shape %s, got %s" % (shape, a.shape))
+    return a
+
+
+def _p(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def rank(x: np.ndarray, p: int) -> int:
+    """rank(p) by counting; p is in the top-k set of x exactly when rank < k (Eq. 2)."""
+    lib = _load()
+    return int(getattr(lib, "oracle_rank_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), x.size, int(p)))
+
+
+def topk(x: np.ndarray, k: int):
+    """Top-k index set of x by magnitude (Eq. 2): returns (idx int32[k] ascending, sel uint8[d])."""
+    lib = _load()
+    d = x.size
+    idx = np.empty(k, np.int32)
+    sel = np.empty(d, np.uint8)
+    rc = getattr(lib, "oracle_topk_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), d, int(k), _p(idx), _p(sel))
+    if rc != 0:
+        raise MemoryError("oracle_topk")
+    return idx, sel
+
+
+def accumulate(g: np.ndarray, m: np.ndarray) -> np.ndarray:
+    """acc = m + g (the argument of CLT-k, Algorithm 1 line 6)."""
+    lib = _load()
+    acc = np.empty_like(g)
+    getattr(lib, "oracle_accumulate_" + _sfx(g.dtype))(_p(_chk(g, g.dtype)), _p(_chk(m, g.dtype, g.shape)), g.size, _p(acc))
+    return acc
+
+
+def learner(g: np.ndarray, m: np.ndarray, idx: np.ndarray, sel: np.ndarray, beta: float) -> np.ndarray:
+    """One learner's gather (Eq. 3) and in-place memory update (Eq. 4); returns gathered[k]."""
+    lib = _load()
+    _chk(m, g.dtype, g.shape); _chk(idx, np.int32); _chk(sel, np.uint8, g.shape)
+    gathered = np.empty(idx.size, g.dtype)
+    getattr(lib, "oracle_learner_" + _sfx(g.dtype))(_p(_chk(g, g.dtype)), _p(m), g.size, _p(idx), idx.size, _p(sel),
+                                                    float(beta), _p(gathered))
+    return gathered
+
+
+def reduce(G: np.ndarray) -> np.ndarray:
+    """val[j] = (sum over learners, in order, of G[i][j]) / n (Algorithm 1 line 10)."""
+    lib = _load()
+    n, k = G.shape
+    val = np.empty(k, G.dtype)
+    getattr(lib, "oracle_reduce_" + _sfx(G.dtype))(_p(_chk(G, G.dtype)), n, k, _p(val))
+    return val
+
+
+def apply(theta: np.ndarray, idx: np.ndarray, val: np.ndarray, lr: float) -> None:
+    """theta[idx[j]] -= lr * val[j], in place (Algorithm 1 line 12)."""
+    lib = _load()
+    _chk(idx, np.int32); _chk(val, theta.dtype, idx.shape)
+    getattr(lib, "oracle_apply_" + _sfx(theta.dtype))(_p(_chk(theta, theta.dtype)), _p(idx), _p(val), idx.size, float(lr))
+
+
+def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: bool = True):
+    """One iteration of Algorithm 1.
+
+    g, m: lists of n ndarrays of d values (m updated in place); theta: ndarray
+    of d values updated in place, or None.  Returns (idx, val, G) with G the
+    n-by-k gathered values (None unless want_gathered).
+    """
+    lib = _load()
+    n = len(g)
+    dtype = g[0].dtype
+    d = g[0].size
+    for a in list(g) + list(m):
+        _chk(a, dtype, (d,))
+    if theta is not None:
+        _chk(theta, dtype, (d,))
+    gp = (ctypes.c_void_p * n)(*[_p(a) for a in g])
+    mp = (ctypes.c_void_p * n)(*[_p(a) for a in m])
+    idx = np.empty(k, np.int32)
+    val = np.empty(k, dtype)
+    G = np.empty((n, k), dtype) if want_gathered else None
+    rc = getattr(lib, "oracle_step_" + _sfx(dtype))(
+        ctypes.cast(gp, ctypes.c_void_p), ctypes.cast(mp, ctypes.c_void_p),
+        _p(theta) if theta is not None else None,
+        int(t), n, d, int(k), float(beta), float(lr), _p(idx), _p(val), _p(G) if G is not None else None)
+    if rc != 0:
+        raise MemoryError("oracle_step")
+    return idx, val, G

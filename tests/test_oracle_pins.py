@@ -1,0 +1,301 @@
+"""Pins for the CPU oracle: every check here compares it with something the
+paper or the mathematics fixes, never with itself and never with the CUDA path."""
+import itertools
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+
+RNG = np.random.default_rng(20210411)
+
+
+def key32(x):
+    return np.ascontiguousarray(x, np.float32).view(np.uint32) & np.uint32(0x7FFFFFFF)
+
+
+def tie_vectors():
+    """Tiny vectors with crafted ties, signed zeros, denormals and +-x pairs."""
+    yield np.array([1, -1, 1, -1, 1, -1, 1, -1], np.float32)
+    yield np.zeros(7, np.float32)
+    yield np.array([0.0, -0.0, 0.0, -0.0, 1e-45, -1e-45], np.float32)
+    yield np.array([3, -3, 2, 2, -2, 1, 5, -5, 5, 0, -0.0, 4], np.float32)
+    yield np.array([2.0], np.float32)
+    for d in (2, 3, 5, 8, 12, 16):
+        yield RNG.integers(-3, 4, size=d).astype(np.float32)          # many ties
+        yield RNG.standard_normal(d).astype(np.float32)               # none
+        yield np.float32(1e-40) * RNG.integers(-2, 3, size=d).astype(np.float32)  # denormals
+
+
+# ---- P1: Eq. 2 by brute force ------------------------------------------------------------
+def test_topk_matches_rank_count_for_all_k():
+    for x in tie_vectors():
+        d = x.size
+        key = key32(x).astype(np.int64)
+        # rank(p) = #{q: key_q > key_p} + #{q < p: key_q == key_p}, counted in Python
+        ranks = [int(sum(1 for q in range(d) if key[q] > key[p] or (key[q] == key[p] and q < p)))
+                 for p in range(d)]
+        assert sorted(ranks) == list(range(d))
+        for p in range(d):
+            assert oracle.rank(x, p) == ranks[p]
+            assert oracle.rank(x.astype(np.float64), p) == ranks[p]
+        for k in range(1, d + 1):
+            idx, sel = oracle.topk(x, k)
+            expect = [p for p in range(d) if ranks[p] < k]
+            assert idx.tolist() == expect
+            assert sel.tolist() == [1 if ranks[p] < k else 0 for p in range(d)]
+            idx64, _ = oracle.topk(x.astype(np.float64), k)
+            assert idx64.tolist() == expect
+
+
+def test_topk_is_the_lexicographically_least_maximiser():
+    """Among all C(d,k) subsets the selected one has the largest total
+    magnitude, and is the first such subset in lexicographic order."""
+    for x in tie_vectors():
+        d = x.size
+        if d > 12:
+            continue
+        mag = [Fraction(float(abs(v))) for v in x.astype(np.float64)]
+        for k in range(1, d + 1):
+            best, best_sum = None, None
+            for S in itertools.combinations(range(d), k):      # lexicographic order
+                s = sum(mag[p] for p in S)
+                if best_sum is None or s > best_sum:
+                    best, best_sum = S, s
+            idx, _ = oracle.topk(x, k)
+            assert tuple(idx.tolist()) == best
+
+
+# ---- exact rational restatement of Algorithm 1 on dyadic inputs ----------------------------
+def _algorithm1_exact(g, m, theta, t, k, beta, lr):
+    """Algorithm 1 in exact rational arithmetic with dense length-d sparse vectors
+    (Eq. 3 literally), valid when every intermediate is exactly representable."""
+    n, d = len(g), len(g[0])
+    L = t % n
+    acc = [[m[i][p] + g[i][p] for p in range(d)] for i in range(n)]
+    order = sorted(range(d), key=lambda p: (-abs(acc[L][p]), p))
+    S = set(order[:k])
+    sparse = [[acc[i][p] if p in S else Fraction(0) for p in range(d)] for i in range(n)]   # Eq. 3
+    new_m = [[(1 - beta) * m[i][p] + beta * (acc[i][p] - sparse[i][p]) for p in range(d)] for i in range(n)]  # Eq. 4
+    gbar = [sum(sparse[i][p] for i in range(n)) / n for p in range(d)]                          # line 10
+    new_theta = [theta[p] - lr * gbar[p] for p in range(d)]                                   # line 12
+    return sorted(S), gbar, sparse, new_m, new_theta
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_step_equals_exact_rational_algorithm1(dtype):
+    rng = np.random.default_rng(7)
+    n, d, k = 4, 24, 5
+    beta, lr = Fraction(1, 4), Fraction(1, 8)
+    g = [[Fraction(int(v), 16) for v in rng.integers(-64, 65, size=d)] for _ in range(n)]
+    m = [[Fraction(int(v), 32) for v in rng.integers(-64, 65, size=d)] for _ in range(n)]
+    theta = [Fraction(int(v), 8) for v in rng.integers(-16, 17, size=d)]
+    for t in range(6):
+        S, gbar, sparse, m2, th2 = _algorithm1_exact(g, m, theta, t, k, beta, lr)
+        gn = [np.array([float(v) for v in row], dtype) for row in g]
+        mn = [np.array([float(v) for v in row], dtype) for row in m]
+        thn = np.array([float(v) for v in theta], dtype)
+        idx, val, G = oracle.step(gn, mn, thn, t, k, float(beta), float(lr))
+        assert idx.tolist() == S
+        assert val.tolist() == [float(gbar[p]) for p in S]
+        for i in range(n):
+            assert G[i].tolist() == [float(sparse[i][p]) for p in S]
+            assert mn[i].tolist() == [float(v) for v in m2[i]]
+        assert thn.tolist() == [float(v) for v in th2]
+        # next iteration: new gradients, carried memory (kept dyadic by beta = 1/4 for a few steps)
+        m, theta = m2, th2
+        g = [[Fraction(int(v), 16) for v in rng.integers(-64, 65, size=d)] for _ in range(n)]
+
+
+# ---- P2: k = d is dense averaged SGD ----------------------------------------------------
+def test_k_equals_d_is_dense_allreduce_sgd():
+    n, d, beta, lr = 5, 257, 0.1, 0.05
+    g = [RNG.standard_normal(d) for _ in range(n)]
+    m = [np.zeros(d) for _ in range(n)]
+    theta = RNG.standard_normal(d)
+    theta0 = theta.copy()
+    idx, val, G = oracle.step(g, m, theta, 3, d, beta, lr)
+    assert idx.tolist() == list(range(d))
+    mean_g = np.mean(np.stack(g), axis=0)
+    np.testing.assert_allclose(val, mean_g, rtol=1e-14, atol=0)
+    np.testing.assert_allclose(theta, theta0 - lr * mean_g, rtol=1e-14, atol=1e-16)
+    for i in range(n):
+        assert not m[i].any()                       # (1-beta)*0 + beta*0
+    # with non-zero memory every coordinate is still sent, so m' = (1-beta) m
+    m = [RNG.standard_normal(d) for _ in range(n)]
+    m0 = [a.copy() for a in m]
+    oracle.step(g, m, None, 0, d, beta, lr)
+    for i in range(n):
+        np.testing.assert_allclose(m[i], (1 - beta) * m0[i], rtol=1e-15)
+
+
+# ---- P3: n = 1, beta = 1 is classical error-feedback top-k (Remark 1) ------------------------
+def test_single_learner_beta_one_is_error_feedback_topk():
+    d, k, lr = 1000, 37, 0.1
+    g = RNG.standard_normal(d).astype(np.float32)
+    m = (0.3 * RNG.standard_normal(d)).astype(np.float32)
+    theta = RNG.standard_normal(d).astype(np.float32)
+    acc = m + g
+    order = np.argsort(-np.abs(acc), kind="stable")[:k]
+    top = np.zeros(d, np.float32)
+    top[order] = acc[order]
+    theta_expect = theta - np.float32(lr) * top
+    m_in = m.copy()
+    idx, val, G = oracle.step([g], [m_in], theta, 11, k, 1.0, lr)
+    assert idx.tolist() == sorted(order.tolist())
+    assert np.array_equal(m_in, acc - top)           # residual, bit for bit
+    assert np.array_equal(theta, theta_expect)
+    assert np.array_equal(val, acc[idx]) and np.array_equal(G[0], acc[idx])
+
+
+# ---- P4: acc = sparse + residual -------------------------------------------------------
+def test_decomposition_identity():
+    n, d, k = 3, 500, 40
+    g = [RNG.standard_normal(d).astype(np.float32) for _ in range(n)]
+    m = [RNG.standard_normal(d).astype(np.float32) for _ in range(n)]
+    acc = [a + b for a, b in zip(m, g)]
+    m1 = [a.copy() for a in m]
+    idx, val, G = oracle.step(g, m1, None, 1, k, 1.0, 0.0)
+    for i in range(n):                                # beta = 1: bitwise
+        sparse = np.zeros(d, np.float32)
+        sparse[idx] = G[i]
+        assert np.array_equal(sparse + m1[i], acc[i])
+        assert not m1[i][idx].any()
+    beta = 0.1                                        # beta < 1 in double
+    g64 = [a.astype(np.float64) for a in g]
+    m64 = [a.astype(np.float64) for a in m]
+    m2 = [a.copy() for a in m64]
+    idx, val, G = oracle.step(g64, m2, None, 1, k, beta, 0.0)
+    for i in range(n):
+        sparse = np.zeros(d)
+        sparse[idx] = G[i]
+        np.testing.assert_allclose((m2[i] - (1 - beta) * m64[i]) / beta + sparse, m64[i] + g64[i],
+                                   rtol=0, atol=1e-12)
+        # a selected coordinate keeps (1-beta) of its memory; it is NOT zeroed unless beta = 1
+        np.testing.assert_allclose(m2[i][idx], (1 - beta) * m64[i][idx], rtol=1e-15)
+
+
+# ---- P5: the leader cycles as t mod n (Algorithm 1 line 6) ---------------------------------
+def test_leader_cycles():
+    n, blk = 4, 16
+    d, k = n * blk, blk
+    g = []
+    for i in range(n):                                # learner i is large exactly on block i
+        v = (0.01 * RNG.standard_normal(d)).astype(np.float32)
+        v[i * blk:(i + 1) * blk] += 10.0
+        g.append(v)
+    seen = []
+    for t in range(3 * n):
+        m = [np.zeros(d, np.float32) for _ in range(n)]
+        idx, _, _ = oracle.step(g, m, None, t, k, 0.5, 0.0)
+        leader = idx[0] // blk
+        assert idx.tolist() == list(range(leader * blk, (leader + 1) * blk))
+        assert leader == t % n
+        seen.append(leader)
+    assert seen[:n] == list(range(n))
+    path = os.path.join(os.path.dirname(__file__), "golden", "leader_demo.txt")
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        gn, gt, gl = map(int, line.split())
+        assert gn == n
+        m = [np.zeros(d, np.float32) for _ in range(n)]
+        idx, _, _ = oracle.step(g, m, None, gt, k, 0.5, 0.0)
+        assert idx[0] // blk == gl
+
+
+# ---- P6: commutativity, Eq. 1 -------------------------------------------------------------
+def test_commutativity_of_cltk_with_averaging():
+    n, d, k, t = 6, 400, 25, 8
+    g = [RNG.standard_normal(d) for _ in range(n)]
+    m = [RNG.standard_normal(d) for _ in range(n)]
+    acc = np.stack([a + b for a, b in zip(m, g)])
+    idx, val, G = oracle.step(g, [a.copy() for a in m], None, t, k, 0.3, 0.0)
+    leader_set, _ = oracle.topk(acc[t % n].copy(), k)
+    assert idx.tolist() == leader_set.tolist()
+    mean_acc = acc.mean(axis=0)
+    lhs = np.zeros(d); lhs[idx] = mean_acc[idx]         # sparse(mean x_i) with the leader's set
+    rhs = np.zeros(d); rhs[idx] = val                   # mean sparse(x_i)
+    np.testing.assert_allclose(lhs, rhs, rtol=1e-13, atol=1e-15)
+    np.testing.assert_array_equal(G, acc[:, idx])
+
+
+# ---- P7: virtual sequence, Appendix D.1 ------------------------------------------------------
+@pytest.mark.parametrize("dtype,tol", [(np.float64, 1e-12), (np.float32, 1e-4)])
+def test_virtual_sequence_identity(dtype, tol):
+    n, d, k, beta, lr, T = 4, 600, 30, 0.1, 0.05, 25
+    theta = np.zeros(d, dtype)                        # theta^0 = v^0 = m^0 = 0
+    v = np.zeros(d, np.float64)
+    m = [np.zeros(d, dtype) for _ in range(n)]
+    rng = np.random.default_rng(3)
+    for t in range(T):
+        g = [rng.standard_normal(d).astype(dtype) for _ in range(n)]
+        v = v - lr * np.mean(np.stack(g).astype(np.float64), axis=0)
+        oracle.step(g, m, theta, t, k, beta, lr)
+        mbar = np.mean(np.stack(m).astype(np.float64), axis=0)
+        lhs = theta.astype(np.float64) - v
+        rhs = (lr / beta) * mbar
+        assert np.max(np.abs(lhs - rhs)) <= tol * max(1.0, np.max(np.abs(rhs)))
+
+
+# ---- P8: contraction, Lemma 1 proof identity and the top-k bound ----------------------------
+def test_contraction_properties():
+    n, d, k, t = 4, 2000, 100, 2
+    g = [RNG.standard_normal(d) for _ in range(n)]
+    m = [np.zeros(d) for _ in range(n)]
+    idx, val, G = oracle.step(g, [a.copy() for a in m], None, t, k, 1.0, 0.0)
+    L = t % n
+    for j in range(n):
+        x = g[j]
+        comp = np.zeros(d); comp[idx] = G[j]
+        lhs = np.sum((x - comp) ** 2)
+        np.testing.assert_allclose(lhs, np.sum(x ** 2) - np.sum(x[idx] ** 2), rtol=1e-12)
+        if j == L:
+            assert lhs <= (1 - k / d) * np.sum(x ** 2)
+
+
+# ---- P9 + P10: threshold property and a library cross-check on a larger vector -----------------
+def test_threshold_property_and_library_topk():
+    d, k = 200_000, 2000
+    x = RNG.standard_normal(d).astype(np.float32)
+    x[RNG.integers(0, d, 500)] = np.float32(2.5)        # a tie group straddling the threshold region
+    idx, sel = oracle.topk(x, k)
+    key = key32(x)
+    assert idx.size == k and np.all(np.diff(idx) > 0)
+    inside, outside = key[sel == 1], key[sel == 0]
+    tau = inside.min()
+    assert tau >= outside.max()
+    ties_in = np.flatnonzero((key == tau) & (sel == 1))
+    ties_out = np.flatnonzero((key == tau) & (sel == 0))
+    if ties_in.size and ties_out.size:
+        assert ties_in.max() < ties_out.min()
+    lib = np.sort(np.argsort(-key.astype(np.int64), kind="stable")[:k])
+    assert np.array_equal(lib, idx)
+    import torch
+    tk = torch.topk(torch.from_numpy(np.abs(x)), k).indices.numpy()
+    strict = key[tk] > tau                               # above the threshold every routine must agree
+    assert set(tk[strict].tolist()) == set(idx[key[idx] > tau].tolist())
+    for p in RNG.integers(0, d, 20):
+        assert (oracle.rank(x, int(p)) < k) == bool(sel[p])
+
+
+def test_pieces_compose_to_step():
+    """The step is exactly accumulate -> topk -> learner x n -> reduce -> apply."""
+    n, d, k, beta, lr, t = 3, 300, 20, 0.1, 0.01, 4
+    g = [RNG.standard_normal(d).astype(np.float32) for _ in range(n)]
+    m = [RNG.standard_normal(d).astype(np.float32) for _ in range(n)]
+    th = RNG.standard_normal(d).astype(np.float32)
+    m1, th1 = [a.copy() for a in m], th.copy()
+    idx, val, G = oracle.step(g, m1, th1, t, k, beta, lr)
+    acc = oracle.accumulate(g[t % n], m[t % n])
+    assert np.array_equal(acc, m[t % n] + g[t % n])
+    idx2, sel = oracle.topk(acc, k)
+    m2 = [a.copy() for a in m]
+    G2 = np.stack([oracle.learner(g[i], m2[i], idx2, sel, beta) for i in range(n)])
+    val2 = oracle.reduce(np.ascontiguousarray(G2))
+    th2 = th.copy()
+    oracle.apply(th2, idx2, val2, lr)
+    assert np.array_equal(idx, idx2) and np.array_equal(val, val2) and np.array_equal(G, G2)
+    assert all(np.array_equal(a, b) for a, b in zip(m1, m2)) and np.array_equal(th1, th2)
