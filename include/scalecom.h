@@ -1,0 +1,171 @@
+/*
+ * scalecom.h -- C ABI of the B200 (sm_100a) CLT-k compression step.
+ *
+ * One call of scalecom_step() is one iteration t of ScaleCom's Algorithm 1 for
+ * n logical learners whose gradients and error-feedback memories live as n + n
+ * fp32 vectors of d values in one GPU's memory:
+ *
+ *   1. acc_i = m_i + g_i                       error feedback, Algorithm 1 line 6
+ *   2. I = top-k index set of |acc_L|,         Eq. 2, leader L = t mod n
+ *      exactly k indices, ties to the lower index, returned ascending
+ *   3. G[i][j] = acc_i[I[j]] (CLT-k, Eq. 3);   val[j] = (G[0][j]+...+G[n-1][j]) / n
+ *      summed in learner order                 Algorithm 1 line 10, Eq. 1
+ *   4. m_i <- (1-beta) m_i + beta (acc_i - CLT-k(acc_i))          Eq. 4
+ *   5. theta[I[j]] <- theta[I[j]] - lr * val[j]                   Algorithm 1 line 12
+ *
+ * Every fp32 operation above is a separately rounded IEEE-754 operation (no
+ * fused multiply-add, no flush to zero), so results do not depend on launch
+ * geometry and are reproducible bit for bit.
+ *
+ * Conventions
+ *   - "DEVICE" pointers address memory of the GPU that was current when the
+ *     handle was created; "HOST" pointers address host memory.
+ *   - All functions return 0 (SCALECOM_OK) or a negative scalecom_error; none
+ *     throws, aborts or traps.  Nothing is launched when an argument is rejected.
+ *   - A handle owns only scratch memory.  All algorithm state (m_i, theta, t)
+ *     belongs to the caller, so a run can be resumed with a fresh handle.
+ *   - A handle is bound to one CUDA stream (default: the legacy default stream);
+ *     calls on one handle must not be made concurrently from several threads.
+ */
+#ifndef SCALECOM_H
+#define SCALECOM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct scalecom_ctx scalecom_ctx;
+
+typedef enum scalecom_error {
+    SCALECOM_OK               = 0,
+    SCALECOM_ERR_INVALID_ARG  = -1,  /* a size or hyper-parameter out of range          */
+    SCALECOM_ERR_NULL_PTR     = -2,  /* a required pointer is NULL                      */
+    SCALECOM_ERR_ALLOC        = -3,  /* host or device allocation failed                */
+    SCALECOM_ERR_CUDA         = -4,  /* a CUDA runtime call or a launch failed          */
+    SCALECOM_ERR_TIMEOUT      = -5,  /* a bounded device-side wait expired              */
+    SCALECOM_ERR_BAD_STATE    = -6,  /* handle poisoned by an earlier device error      */
+    SCALECOM_ERR_INTERNAL     = -7,  /* a device-side consistency check failed          */
+    SCALECOM_ERR_ALIAS        = -8   /* buffers that must be distinct overlap           */
+} scalecom_error;
+
+/* Largest number of learners one handle accepts (pointer tables travel as kernel arguments). */
+#define SCALECOM_MAX_LEARNERS 1024
+
+/*
+ * Create a handle for vectors of d coordinates, n learners and k kept
+ * coordinates (Algorithm 1's inputs; 0 < beta <= 1 is Eq. 4's discounting
+ * factor, lr is the step size alpha of line 12).
+ *   out    HOST, receives the handle.
+ *   d      1 <= d <= 2^31 - 1.      n   1 <= n <= SCALECOM_MAX_LEARNERS.
+ *   k      1 <= k <= d.             beta in (0, 1].   lr finite.
+ * Allocates the scratch workspace (about d/8 + 24k + 1 MB bytes) on the current
+ * device with cudaMalloc.  Errors: INVALID_ARG, NULL_PTR, ALLOC, CUDA.
+ */
+int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float beta, float lr);
+
+/*
+ * One iteration of Algorithm 1 (steps 1-5 above), asynchronous on the handle's
+ * stream: no host synchronisation, no device-to-host copy.
+ *   grads    HOST array of n DEVICE pointers, each fp32[d], read only.
+ *   mem      HOST array of n DEVICE pointers, each fp32[d], updated in place (Eq. 4).
+ *   weights  DEVICE fp32[d], updated in place at the k selected coordinates;
+ *            NULL skips step 5 (the caller applies its own optimiser to out_val).
+ *   t        iteration index >= 0; the leader is learner t mod n.
+ *   out_idx  DEVICE int32[k], written: the selected coordinates, ascending.
+ *   out_val  DEVICE fp32[k], written: the averaged reduced values at out_idx.
+ * The two pointer arrays are read during the call and may be reused at once.
+ * grads[i], mem[i], weights and the outputs must not overlap one another
+ * (exact pointer equality is rejected with ALIAS; partial overlap is undefined).
+ * Any alignment is accepted; 16-byte aligned vectors take the fast path.
+ * Errors: NULL_PTR, INVALID_ARG (t < 0), ALIAS, BAD_STATE, CUDA.
+ */
+int scalecom_step(scalecom_ctx* ctx,
+                  const float* const* grads,
+                  float* const* mem,
+                  float* weights,
+                  int64_t t,
+                  int32_t* out_idx,
+                  float* out_val);
+
+/*
+ * The same iteration for callers whose gradients and results live in HOST
+ * memory (Algorithm 1 lines 9 and 11, "upload"/"download"): copies the n
+ * gradients to a device staging area owned by the handle (allocated on first
+ * use, n*d*4 bytes), runs scalecom_step, copies out_idx and out_val back and
+ * waits for the stream.  mem and weights stay DEVICE pointers (they are state,
+ * not per-iteration traffic).  Pinned host memory makes the copies asynchronous.
+ *   host_grads  HOST array of n HOST pointers, each fp32[d].
+ *   host_idx    HOST int32[k], written.     host_val  HOST fp32[k], written.
+ * Errors: as scalecom_step, plus ALLOC.
+ */
+int scalecom_step_host(scalecom_ctx* ctx,
+                       const float* const* host_grads,
+                       float* const* mem,
+                       float* weights,
+                       int64_t t,
+                       int32_t* host_idx,
+                       float* host_val);
+
+/* Release the workspace.  NULL is accepted.  Synchronises the handle's stream first. */
+void scalecom_destroy(scalecom_ctx* ctx);
+
+/* Bind the handle to a CUDA stream (a cudaStream_t passed as void*; NULL = legacy default). */
+int scalecom_set_stream(scalecom_ctx* ctx, void* cuda_stream);
+
+/*
+ * Ask every later step to also write the per-learner gathered values of Eq. 3:
+ * G[i*k + j] = acc_i[out_idx[j]] into the caller's DEVICE fp32[n*k] buffer.
+ * NULL (the default) turns the extra output off.
+ */
+int scalecom_set_gathered(scalecom_ctx* ctx, float* dev_gathered);
+
+/*
+ * Algorithm 1 line 12 on its own: theta[idx[j]] <- theta[idx[j]] - lr * val[j]
+ * for j < k, on the handle's stream, for callers that ran scalecom_step with
+ * weights == NULL.  All pointers DEVICE; idx entries must be distinct and < d.
+ */
+int scalecom_apply_update(scalecom_ctx* ctx, float* weights, const int32_t* idx,
+                          const float* val, int64_t k, float lr);
+
+/*
+ * Wait for the handle's stream and report the device-side status of the steps
+ * issued so far: SCALECOM_OK, SCALECOM_ERR_TIMEOUT or SCALECOM_ERR_INTERNAL
+ * (after either of which outputs are undefined and the handle refuses further
+ * steps until scalecom_reset), or SCALECOM_ERR_CUDA.
+ */
+int scalecom_status(scalecom_ctx* ctx);
+
+/* Clear a device-side error and re-initialise the workspace (synchronises). */
+int scalecom_reset(scalecom_ctx* ctx);
+
+/* Options for scalecom_set_option. */
+#define SCALECOM_OPT_FORCE_EXACT_PATH 1  /* 1: skip the sampled pre-filter, always run the full radix select */
+#define SCALECOM_OPT_SPIN_LIMIT       2  /* iteration bound of the in-kernel grid barrier wait (>= 0)       */
+#define SCALECOM_OPT_KERNEL_TIMING    3  /* 1: bracket each kernel of a step with CUDA events                */
+#define SCALECOM_OPT_FUSE_UPDATE      4  /* 1 (default): step 5 runs inside the learner pass; 0: own kernel  */
+int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
+
+/* Items for scalecom_query (each synchronises the stream when it reads device state). */
+#define SCALECOM_Q_WORKSPACE_BYTES  1  /* device bytes owned by the handle                                    */
+#define SCALECOM_Q_LAST_TOPK_PATH   2  /* last step's selection path: 0 = sampled pre-filter, 1 = full select */
+#define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
+#define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
+#define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */
+int scalecom_query(scalecom_ctx* ctx, int item, int64_t* out);
+
+/*
+ * With SCALECOM_OPT_KERNEL_TIMING on: waits for the last step and writes its
+ * kernel durations in milliseconds: ms[0] selection (step 2), ms[1] learner
+ * pass (steps 1, 3, 4, and 5 when fused), ms[2] separate weight update (0 when fused).
+ */
+int scalecom_last_kernel_ms(scalecom_ctx* ctx, float ms[3]);
+
+/* Static, never NULL. */
+const char* scalecom_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCALECOM_H */

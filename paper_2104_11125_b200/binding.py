@@ -1,0 +1,216 @@
+"""ctypes binding of libscalecom.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name in
+include/scalecom.h; torch is used for device memory and streams, nothing is
+computed here.  There is no fallback: if the compiled library is missing the
+first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libscalecom.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_NULL_PTR, ERR_ALLOC, ERR_CUDA = -1, -2, -3, -4
+ERR_TIMEOUT, ERR_BAD_STATE, ERR_INTERNAL, ERR_ALIAS = -5, -6, -7, -8
+MAX_LEARNERS = 1024
+
+OPT_FORCE_EXACT_PATH, OPT_SPIN_LIMIT, OPT_KERNEL_TIMING, OPT_FUSE_UPDATE = 1, 2, 3, 4
+Q_WORKSPACE_BYTES, Q_LAST_TOPK_PATH, Q_LAST_CANDIDATES, Q_TOPK_BLOCKS, Q_KERNEL_LAUNCHES = 1, 2, 3, 4, 5
+
+EXPORTS = (
+    "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
+    "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
+    "scalecom_set_option", "scalecom_query", "scalecom_last_kernel_ms", "scalecom_strerror",
+)
+
+_lib = None
+
+
+class ScaleComError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (%d)" % (where, strerror(code), code))
+
+
+def lib() -> ctypes.CDLL:
+    """Load the compiled library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libscalecom.so is missing (%s): build it with "
+                "`python -m paper_2104_11125_b200.build`; there is no fallback path" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+        L.scalecom_create.restype = ctypes.c_int
+        L.scalecom_create.argtypes = [ctypes.POINTER(vp), i64, i32, i64, f32, f32]
+        L.scalecom_step.restype = ctypes.c_int
+        L.scalecom_step.argtypes = [vp, vp, vp, vp, i64, vp, vp]
+        L.scalecom_step_host.restype = ctypes.c_int
+        L.scalecom_step_host.argtypes = [vp, vp, vp, vp, i64, vp, vp]
+        L.scalecom_destroy.restype = None
+        L.scalecom_destroy.argtypes = [vp]
+        L.scalecom_set_stream.restype = ctypes.c_int
+        L.scalecom_set_stream.argtypes = [vp, vp]
+        L.scalecom_set_gathered.restype = ctypes.c_int
+        L.scalecom_set_gathered.argtypes = [vp, vp]
+        L.scalecom_apply_update.restype = ctypes.c_int
+        L.scalecom_apply_update.argtypes = [vp, vp, vp, vp, i64, f32]
+        L.scalecom_status.restype = ctypes.c_int
+        L.scalecom_status.argtypes = [vp]
+        L.scalecom_reset.restype = ctypes.c_int
+        L.scalecom_reset.argtypes = [vp]
+        L.scalecom_set_option.restype = ctypes.c_int
+        L.scalecom_set_option.argtypes = [vp, ctypes.c_int, i64]
+        L.scalecom_query.restype = ctypes.c_int
+        L.scalecom_query.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64)]
+        L.scalecom_last_kernel_ms.restype = ctypes.c_int
+        L.scalecom_last_kernel_ms.argtypes = [vp, ctypes.POINTER(f32)]
+        L.scalecom_strerror.restype = ctypes.c_char_p
+        L.scalecom_strerror.argtypes = [ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().scalecom_strerror(int(code)).decode()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise ScaleComError(rc, where)
+
+
+# ---- raw mirrors of the C entry points (integers in, return codes out) -------------------------
+def scalecom_create(d: int, n: int, k: int, beta: float, lr: float) -> Tuple[int, Optional[int]]:
+    h = ctypes.c_void_p()
+    rc = lib().scalecom_create(ctypes.byref(h), int(d), int(n), int(k), float(beta), float(lr))
+    return rc, h.value
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    return (ctypes.c_void_p * len(ptrs))(*ptrs)
+
+
+def scalecom_step(handle: int, grads: Sequence[int], mem: Sequence[int], weights: Optional[int], t: int,
+                  out_idx: int, out_val: int) -> int:
+    ga, ma = _ptr_array(grads), _ptr_array(mem)
+    return lib().scalecom_step(handle, ctypes.cast(ga, ctypes.c_void_p), ctypes.cast(ma, ctypes.c_void_p),
+                               weights, int(t), out_idx, out_val)
+
+
+def scalecom_step_host(handle: int, host_grads: Sequence[int], mem: Sequence[int], weights: Optional[int], t: int,
+                       host_idx: int, host_val: int) -> int:
+    ga, ma = _ptr_array(host_grads), _ptr_array(mem)
+    return lib().scalecom_step_host(handle, ctypes.cast(ga, ctypes.c_void_p), ctypes.cast(ma, ctypes.c_void_p),
+                                    weights, int(t), host_idx, host_val)
+
+
+def scalecom_destroy(handle: Optional[int]) -> None:
+    lib().scalecom_destroy(handle)
+
+
+# ---- tensor-level convenience wrapper ------------------------------------------------------------
+def _dev_f32(t: torch.Tensor, numel: int, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+            and t.numel() == numel):
+        raise TypeError("%s must be a contiguous CUDA float32 tensor of %d elements" % (name, numel))
+    return t.data_ptr()
+
+
+class Context:
+    """One scalecom handle.  State (memories, weights, t) stays with the caller."""
+
+    def __init__(self, d: int, n: int, k: int, beta: float, lr: float, stream: Optional[torch.cuda.Stream] = None):
+        self.d, self.n, self.k, self.beta, self.lr = int(d), int(n), int(k), float(beta), float(lr)
+        rc, h = scalecom_create(d, n, k, beta, lr)
+        _check(rc, "scalecom_create")
+        self._h = h
+        self._gathered = None
+        if stream is not None:
+            self.set_stream(stream)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            scalecom_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def set_stream(self, stream: Optional[torch.cuda.Stream]) -> None:
+        _check(lib().scalecom_set_stream(self._h, stream.cuda_stream if stream is not None else None),
+               "scalecom_set_stream")
+
+    def set_gathered(self, buf: Optional[torch.Tensor]) -> None:
+        ptr = None if buf is None else _dev_f32(buf, self.n * self.k, "gathered")
+        _check(lib().scalecom_set_gathered(self._h, ptr), "scalecom_set_gathered")
+        self._gathered = buf
+
+    def set_option(self, option: int, value: int) -> None:
+        _check(lib().scalecom_set_option(self._h, option, int(value)), "scalecom_set_option")
+
+    def query(self, item: int) -> int:
+        out = ctypes.c_int64()
+        _check(lib().scalecom_query(self._h, item, ctypes.byref(out)), "scalecom_query")
+        return out.value
+
+    def status(self) -> int:
+        return lib().scalecom_status(self._h)
+
+    def reset(self) -> None:
+        _check(lib().scalecom_reset(self._h), "scalecom_reset")
+
+    def last_kernel_ms(self) -> List[float]:
+        ms = (ctypes.c_float * 3)()
+        _check(lib().scalecom_last_kernel_ms(self._h, ms), "scalecom_last_kernel_ms")
+        return list(ms)
+
+    def step(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], weights: Optional[torch.Tensor],
+             t: int, out_idx: torch.Tensor, out_val: torch.Tensor) -> None:
+        """scalecom_step on device tensors (asynchronous on the handle's stream)."""
+        if len(grads) != self.n or len(mem) != self.n:
+            raise ValueError("expected %d gradient and %d memory tensors" % (self.n, self.n))
+        gp = [_dev_f32(g, self.d, "grads[%d]" % i) for i, g in enumerate(grads)]
+        mp = [_dev_f32(m, self.d, "mem[%d]" % i) for i, m in enumerate(mem)]
+        wp = None if weights is None else _dev_f32(weights, self.d, "weights")
+        if not (out_idx.is_cuda and out_idx.dtype == torch.int32 and out_idx.is_contiguous() and out_idx.numel() == self.k):
+            raise TypeError("out_idx must be a contiguous CUDA int32 tensor of k elements")
+        _check(scalecom_step(self._h, gp, mp, wp, t, out_idx.data_ptr(), _dev_f32(out_val, self.k, "out_val")),
+               "scalecom_step")
+
+    def step_host(self, host_grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor],
+                  weights: Optional[torch.Tensor], t: int, host_idx: torch.Tensor, host_val: torch.Tensor) -> None:
+        """scalecom_step_host: gradients and results in host tensors (synchronous)."""
+        if len(host_grads) != self.n or len(mem) != self.n:
+            raise ValueError("expected %d gradient and %d memory tensors" % (self.n, self.n))
+        for i, g in enumerate(host_grads):
+            if g.is_cuda or g.dtype != torch.float32 or not g.is_contiguous() or g.numel() != self.d:
+                raise TypeError("host_grads[%d] must be a contiguous CPU float32 tensor of d elements" % i)
+        if host_idx.is_cuda or host_idx.dtype != torch.int32 or host_idx.numel() != self.k or not host_idx.is_contiguous():
+            raise TypeError("host_idx must be a contiguous CPU int32 tensor of k elements")
+        if host_val.is_cuda or host_val.dtype != torch.float32 or host_val.numel() != self.k or not host_val.is_contiguous():
+            raise TypeError("host_val must be a contiguous CPU float32 tensor of k elements")
+        mp = [_dev_f32(m, self.d, "mem[%d]" % i) for i, m in enumerate(mem)]
+        wp = None if weights is None else _dev_f32(weights, self.d, "weights")
+        _check(scalecom_step_host(self._h, [g.data_ptr() for g in host_grads], mp, wp, t,
+                                  host_idx.data_ptr(), host_val.data_ptr()), "scalecom_step_host")
+
+    def apply_update(self, weights: torch.Tensor, idx: torch.Tensor, val: torch.Tensor, lr: float) -> None:
+        k = idx.numel()
+        if not (idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous()):
+            raise TypeError("idx must be a contiguous CUDA int32 tensor")
+        _check(lib().scalecom_apply_update(self._h, _dev_f32(weights, self.d, "weights"), idx.data_ptr(),
+                                           _dev_f32(val, k, "val"), k, float(lr)), "scalecom_apply_update")

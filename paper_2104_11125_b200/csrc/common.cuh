@@ -1,0 +1,111 @@
+// Shared device helpers of the CLT-k kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sc {
+
+// Device-side status codes (mirrors of the negative C-ABI errors, stored positive).
+constexpr uint32_t DEV_OK = 0;
+constexpr uint32_t DEV_TIMEOUT = 5;
+constexpr uint32_t DEV_INTERNAL = 7;
+
+// Coordinates per tile of the learner pass; one tile owns 32 words of the selection bitmap.
+constexpr uint32_t TILE = 1024;
+
+constexpr unsigned FULL = 0xFFFFFFFFu;
+
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }
+__device__ __forceinline__ uint32_t warp_id() { return threadIdx.x >> 5; }
+
+// Magnitude key of Eq. 2: the bit pattern of |x|; unsigned order == magnitude order.
+__device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+// Total order "larger magnitude first, then lower index first" as one 62-bit
+// number: larger composite == earlier in that order; all composites are distinct.
+__device__ __forceinline__ uint64_t composite(uint32_t key, uint32_t idx) {
+    return (uint64_t(key) << 31) | uint64_t(0x7FFFFFFFu - idx);
+}
+
+// ---- streaming loads / stores ---------------------------------------------------------------
+// Four consecutive coordinates starting at p.  VEC: one 128-bit load when the
+// quad is fully inside [0, d); otherwise (ragged tail, or unaligned vectors)
+// guarded scalar loads that return 0 beyond d.
+template <bool VEC>
+__device__ __forceinline__ void load_quad_stream(const float* __restrict__ a, uint32_t p, uint32_t d, float (&v)[4]) {
+    if (VEC && p + 4u <= d) {
+        const float4 t = __ldcs(reinterpret_cast<const float4*>(a + p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] = (p + c < d) ? __ldcs(a + p + c) : 0.0f;
+    }
+}
+
+template <bool VEC>
+__device__ __forceinline__ void store_quad_stream(float* __restrict__ a, uint32_t p, uint32_t d, const float (&v)[4]) {
+    if (VEC && p + 4u <= d) {
+        __stcs(reinterpret_cast<float4*>(a + p), make_float4(v[0], v[1], v[2], v[3]));
+    } else {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (p + c < d) __stcs(a + p + c, v[c]);
+    }
+}
+
+// ---- warp scans -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(FULL, v, o);
+        if (lane_id() >= (uint32_t)o) v += t;
+    }
+    return v;
+}
+
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+    return v;
+}
+
+// ---- bounded grid barrier ----------------------------------------------------------------------
+// All blocks of a cooperative launch call this the same number of times.  The
+// 64-bit counter only ever grows; each arrival derives its own release value, so
+// no reset between barriers or launches is needed as long as every launch
+// completes (the host zeroes the counter after a device error).  The wait is
+// bounded: on expiry the status word becomes DEV_TIMEOUT, every waiter sees it
+// and the function returns false; callers then return without touching memory.
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ bool grid_barrier(unsigned long long* counter, uint32_t nblocks,
+                                             uint32_t* status, uint32_t spin_limit, int* smem_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ok = 0;
+        __threadfence();
+        const unsigned long long old = atomicAdd(counter, 1ULL);
+        const unsigned long long target = (old / nblocks + 1ULL) * nblocks;
+        for (uint32_t it = 0; it <= spin_limit; ++it) {
+            if (ld_acquire_u64(counter) >= target) { ok = 1; break; }
+            if (ld_relaxed_u32(status) != DEV_OK) break;
+            if (it > 64) __nanosleep(it > 4096 ? 256 : 32);
+        }
+        if (!ok) atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+        __threadfence();
+        *smem_flag = ok;
+    }
+    __syncthreads();
+    return *smem_flag != 0;
+}
+
+}  // namespace sc

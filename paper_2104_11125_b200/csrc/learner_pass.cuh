@@ -1,0 +1,111 @@
+// Fused learner pass: Algorithm 1 lines 6-7 and 10 (and 12) for all n learners
+// in one streaming sweep.  Every g_i and m_i is read once and m_i written once
+// (12 bytes per learner-coordinate); acc_i = m_i + g_i is never stored.
+//
+// Work is cut by coordinate, not by learner: a tile of 1024 coordinates is
+// owned by one block, each thread keeps its four coordinates for all learners,
+// so the cross-learner sum of Algorithm 1 line 10 is a register accumulation
+// in learner order 0..n-1 -- no atomics, no second pass, bitwise reproducible.
+// Whether a coordinate is selected comes from the leader's bitmap; its rank in
+// the ascending index list (where the gathered and reduced values go) from the
+// per-tile prefix counts written by the selection kernel.
+#pragma once
+#include "common.cuh"
+
+namespace sc {
+
+constexpr int LP_THREADS = 256;            // x 4 coordinates = one tile
+constexpr int LP_UNROLL = 4;               // learners in flight per thread
+
+template <int N>
+struct PtrTable {
+    const float* g[N];
+    float* m[N];
+};
+
+struct LearnerParams {
+    uint32_t d, k, ntiles;
+    int32_t n;
+    float beta, omb, lr, nf;               // omb = 1 - beta rounded once in fp32; nf = (float)n
+    const uint32_t* bitmap;                // [ntiles * 32]
+    const uint32_t* tile_prefix;           // [ntiles + 1]
+    float* out_val;                        // [k]
+    float* gathered;                       // [n * k] or nullptr
+    float* weights;                        // [d] or nullptr (then Algorithm 1 line 12 is not applied here)
+};
+
+template <int N, bool VEC>
+__global__ void __launch_bounds__(LP_THREADS, 4)
+learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P) {
+    const uint32_t tid = threadIdx.x, lane = lane_id();
+    const uint32_t d = P.d;
+    const int n = P.n;
+    const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside the tile
+    const uint32_t sh = (tid & 7u) * 4u;           // and its first bit inside that word
+
+    for (uint32_t tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
+        // selection bits of this thread's four coordinates and the rank of the first selected one
+        const uint32_t w = __ldg(&P.bitmap[size_t(tile) * 32 + lane]);
+        const uint32_t cnt = __popc(w);
+        const uint32_t incl = warp_incl_scan(cnt);
+        const uint32_t excl_word = __shfl_sync(FULL, incl - cnt, wi);
+        const uint32_t myword = __shfl_sync(FULL, w, wi);
+        const uint32_t nib = (myword >> sh) & 15u;
+        const uint32_t rank0 = __ldg(&P.tile_prefix[tile]) + excl_word + __popc(myword & ((1u << sh) - 1u));
+
+        const uint32_t p = tile * TILE + tid * 4u;
+        if (p >= d) continue;
+
+        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int i0 = 0; i0 < n; i0 += LP_UNROLL) {
+            float gv[LP_UNROLL][4], mv[LP_UNROLL][4];
+#pragma unroll
+            for (int u = 0; u < LP_UNROLL; ++u)
+                if (i0 + u < n) {
+                    load_quad_stream<VEC>(tab.g[i0 + u], p, d, gv[u]);
+                    load_quad_stream<VEC>(tab.m[i0 + u], p, d, mv[u]);
+                }
+#pragma unroll
+            for (int u = 0; u < LP_UNROLL; ++u)
+                if (i0 + u < n) {
+                    const int i = i0 + u;
+                    float acc[4], out[4];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        acc[c] = __fadd_rn(mv[u][c], gv[u][c]);                        // line 6: m + g
+                        sum[c] = (i == 0) ? acc[c] : __fadd_rn(sum[c], acc[c]);       // line 10, learner order
+                        const float r = ((nib >> c) & 1u) ? 0.0f : acc[c];            // acc - CLT-k(acc)
+                        out[c] = __fadd_rn(__fmul_rn(P.omb, mv[u][c]), __fmul_rn(P.beta, r));   // Eq. 4
+                    }
+                    store_quad_stream<VEC>(tab.m[i], p, d, out);
+                    if (nib && P.gathered) {                                           // Eq. 3: learner i's kept values
+                        uint32_t r = rank0;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            if ((nib >> c) & 1u) P.gathered[size_t(i) * P.k + r++] = acc[c];
+                    }
+                }
+        }
+        if (nib) {
+            uint32_t r = rank0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if ((nib >> c) & 1u) {
+                    const float v = __fdiv_rn(sum[c], P.nf);                           // line 10: one division by n
+                    P.out_val[r++] = v;
+                    if (P.weights) P.weights[p + c] = __fsub_rn(P.weights[p + c], __fmul_rn(P.lr, v));   // line 12
+                }
+        }
+    }
+}
+
+// Algorithm 1 line 12 as its own kernel: theta[idx[j]] -= lr * val[j].
+__global__ void __launch_bounds__(256) apply_update_kernel(float* __restrict__ weights, const int32_t* __restrict__ idx,
+                                                           const float* __restrict__ val, uint32_t k, float lr) {
+    for (uint32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < k; j += gridDim.x * blockDim.x) {
+        const int32_t p = idx[j];
+        weights[p] = __fsub_rn(weights[p], __fmul_rn(lr, val[j]));
+    }
+}
+
+}  // namespace sc

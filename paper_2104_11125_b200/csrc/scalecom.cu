@@ -1,0 +1,485 @@
+// C-ABI of the CLT-k step (see include/scalecom.h): argument checks, workspace, launches.
+#include "../../include/scalecom.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "learner_pass.cuh"
+#include "topk_select.cuh"
+
+using namespace sc;
+
+struct scalecom_ctx {
+    int device = 0;
+    int64_t d = 0, k = 0;
+    int32_t n = 0;
+    float beta = 0.f, lr = 0.f;
+    cudaStream_t stream = nullptr;
+
+    // workspace (one allocation)
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    uint32_t *samp_hist = nullptr, *coarse_win = nullptr, *fine_hist = nullptr, *digit_hist = nullptr;
+    uint32_t *block_tot = nullptr, *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr;
+    unsigned long long* barrier = nullptr;
+    uint2* cand = nullptr;
+    uint32_t cand_cap = 0, ntiles = 0, tiles_per_block = 0;
+    size_t ctrl_region_bytes = 0;      // prefix of the workspace that reset() clears
+
+    // launch geometry
+    int sms = 0;
+    uint32_t topk_blocks = 0, lp_blocks = 0;
+    uint32_t samp_stride = 1, samp_target = 1;
+
+    // options
+    uint32_t force_exact = 0;
+    uint32_t spin_limit = 1u << 22;
+    bool timing = false;
+    bool fuse_update = true;
+    float* gathered = nullptr;
+
+    // host-buffer entry point
+    float* stage_g = nullptr;          // n*d
+    int32_t* stage_idx = nullptr;      // k
+    float* stage_val = nullptr;        // k
+
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool ev_valid = false;
+    bool poisoned = false;
+    int64_t launches = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <bool VEC>
+cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
+    void* args[] = {const_cast<TopkParams*>(&P)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&topk_select_kernel<VEC>), dim3(c->topk_blocks),
+                                       dim3(TK_THREADS), args, sizeof(TopkShared), c->stream);
+}
+
+template <int N, bool VEC>
+cudaError_t launch_learner(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
+    PtrTable<N> tab;
+    for (int i = 0; i < N; ++i) {
+        tab.g[i] = i < c->n ? grads[i] : nullptr;
+        tab.m[i] = i < c->n ? mem[i] : nullptr;
+    }
+    learner_pass_kernel<N, VEC><<<c->lp_blocks, LP_THREADS, 0, c->stream>>>(tab, P);
+    return cudaGetLastError();
+}
+
+template <bool VEC>
+cudaError_t launch_learner_n(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
+    if (c->n <= 16) return launch_learner<16, VEC>(c, grads, mem, P);
+    if (c->n <= 128) return launch_learner<128, VEC>(c, grads, mem, P);
+    return launch_learner<SCALECOM_MAX_LEARNERS, VEC>(c, grads, mem, P);
+}
+
+int init_workspace(scalecom_ctx* c) {
+    if (cudaMemsetAsync(c->ws, 0, c->ctrl_region_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    return SCALECOM_OK;
+}
+
+int check_step_args(scalecom_ctx* c, const void* const* grads, const void* const* mem, const void* weights, int64_t t,
+                    const void* out_idx, const void* out_val) {
+    if (!c || !grads || !mem || !out_idx || !out_val) return SCALECOM_ERR_NULL_PTR;
+    if (t < 0) return SCALECOM_ERR_INVALID_ARG;
+    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
+    for (int i = 0; i < c->n; ++i)
+        if (!grads[i] || !mem[i]) return SCALECOM_ERR_NULL_PTR;
+    if (out_idx == out_val || out_idx == weights || out_val == weights) return SCALECOM_ERR_ALIAS;
+    for (int i = 0; i < c->n; ++i) {
+        const void* a[2] = {grads[i], mem[i]};
+        for (const void* x : a)
+            if (x == weights || x == out_idx || x == out_val) return SCALECOM_ERR_ALIAS;
+        if (grads[i] == mem[i]) return SCALECOM_ERR_ALIAS;
+    }
+    if (c->n <= 64) {            // quadratic check only where it is cheap; mem buffers are written, so they must be distinct
+        for (int i = 0; i < c->n; ++i)
+            for (int j = 0; j < c->n; ++j) {
+                if (i != j && mem[i] == mem[j]) return SCALECOM_ERR_ALIAS;
+                if (grads[i] == mem[j]) return SCALECOM_ERR_ALIAS;
+            }
+    }
+    return SCALECOM_OK;
+}
+
+int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float* weights, int64_t t, int32_t* out_idx,
+            float* out_val) {
+    const int leader = int(t % c->n);
+
+    TopkParams tp;
+    tp.g = grads[leader];
+    tp.m = mem[leader];
+    tp.d = uint32_t(c->d);
+    tp.k = uint32_t(c->k);
+    tp.samp_stride = c->samp_stride;
+    tp.samp_target = c->samp_target;
+    tp.force_exact = c->force_exact;
+    tp.spin_limit = c->spin_limit;
+    tp.samp_hist = c->samp_hist;
+    tp.coarse_win = c->coarse_win;
+    tp.fine_hist = c->fine_hist;
+    tp.digit_hist = c->digit_hist;
+    tp.block_tot = c->block_tot;
+    tp.ctrl = c->ctrl;
+    tp.barrier = c->barrier;
+    tp.cand = c->cand;
+    tp.cand_cap = c->cand_cap;
+    tp.bitmap = c->bitmap;
+    tp.tile_prefix = c->tile_prefix;
+    tp.ntiles = c->ntiles;
+    tp.tiles_per_block = c->tiles_per_block;
+    tp.out_idx = out_idx;
+
+    LearnerParams lp;
+    lp.d = uint32_t(c->d);
+    lp.k = uint32_t(c->k);
+    lp.ntiles = c->ntiles;
+    lp.n = c->n;
+    lp.beta = c->beta;
+    lp.omb = 1.0f - c->beta;
+    lp.lr = c->lr;
+    lp.nf = float(c->n);
+    lp.bitmap = c->bitmap;
+    lp.tile_prefix = c->tile_prefix;
+    lp.out_val = out_val;
+    lp.gathered = c->gathered;
+    lp.weights = (weights && c->fuse_update) ? weights : nullptr;
+
+    bool vec_all = true;
+    for (int i = 0; i < c->n; ++i) vec_all = vec_all && aligned16(grads[i]) && aligned16(mem[i]);
+    const bool vec_leader = aligned16(tp.g) && aligned16(tp.m);
+
+    const bool tm = c->timing;
+    if (tm && cudaEventRecord(c->ev[0], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    cudaError_t e = vec_leader ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
+    if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
+    ++c->launches;
+    if (tm && cudaEventRecord(c->ev[1], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    e = vec_all ? launch_learner_n<true>(c, grads, mem, lp) : launch_learner_n<false>(c, grads, mem, lp);
+    if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
+    ++c->launches;
+    if (tm && cudaEventRecord(c->ev[2], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (weights && !c->fuse_update) {
+        const uint32_t blocks = uint32_t((c->k + 255) / 256);
+        apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, out_idx, out_val,
+                                                                                   uint32_t(c->k), c->lr);
+        if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+        ++c->launches;
+    }
+    if (tm) {
+        if (cudaEventRecord(c->ev[3], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+        c->ev_valid = true;
+    }
+    return SCALECOM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float beta, float lr) {
+    if (!out) return SCALECOM_ERR_NULL_PTR;
+    *out = nullptr;
+    if (d < 1 || d > 2147483647LL || n < 1 || n > SCALECOM_MAX_LEARNERS || k < 1 || k > d) return SCALECOM_ERR_INVALID_ARG;
+    if (!(beta > 0.0f) || !(beta <= 1.0f) || !std::isfinite(lr)) return SCALECOM_ERR_INVALID_ARG;
+
+    scalecom_ctx* c = new (std::nothrow) scalecom_ctx;
+    if (!c) return SCALECOM_ERR_ALLOC;
+    c->d = d; c->n = n; c->k = k; c->beta = beta; c->lr = lr;
+
+    int coop = 0, occ_topk = 0, occ_lp = 0;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(topk_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(TopkShared)));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(topk_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(TopkShared)));
+    if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_topk, topk_select_kernel<true>, TK_THREADS, sizeof(TopkShared));
+    if (e == cudaSuccess) {
+        int o2 = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o2, topk_select_kernel<false>, TK_THREADS, sizeof(TopkShared));
+        if (o2 < occ_topk) occ_topk = o2;
+    }
+    if (e == cudaSuccess)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_lp, learner_pass_kernel<16, true>, LP_THREADS, 0);
+    if (e != cudaSuccess || !coop || occ_topk < 1 || occ_lp < 1) {
+        cudaGetLastError();
+        delete c;
+        return SCALECOM_ERR_CUDA;
+    }
+    if (occ_topk > 2) occ_topk = 2;
+
+    c->ntiles = uint32_t((d + TILE - 1) / TILE);
+    // persistent selection grid: every resident slot, but no more blocks than there are chunks of work
+    const uint32_t chunks = uint32_t((d + TK_CHUNK - 1) / TK_CHUNK);
+    c->topk_blocks = uint32_t(c->sms * occ_topk);
+    if (c->topk_blocks > chunks) c->topk_blocks = chunks;
+    if (c->topk_blocks < 1) c->topk_blocks = 1;
+    c->tiles_per_block = (c->ntiles + c->topk_blocks - 1) / c->topk_blocks;
+    c->lp_blocks = uint32_t(c->sms * occ_lp);
+    if (c->lp_blocks > c->ntiles) c->lp_blocks = c->ntiles;
+
+    // sampling rate: about 2^18 sampled keys or 1/64 of the vector, whichever is more
+    uint32_t stride = 1;
+    while (stride < 64 && (d / (2 * stride)) >= (1 << 18)) stride *= 2;
+    c->samp_stride = stride;
+    {
+        const int64_t span = int64_t(SAMPLE_GRANULE) * stride;
+        const int64_t full = d / span, rem = d % span;
+        const int64_t ns = full * SAMPLE_GRANULE + (rem < SAMPLE_GRANULE ? rem : SAMPLE_GRANULE);
+        if (stride == 1) {
+            c->samp_target = uint32_t(k);                                  // the "sample" is the whole vector: exact bin
+        } else {
+            const double ks = double(k) * double(ns) / double(d);
+            double tgt = std::ceil(ks + 6.0 * std::sqrt(ks) + 8.0);
+            if (tgt > double(ns)) tgt = double(ns);
+            c->samp_target = uint32_t(tgt);
+        }
+    }
+    {
+        int64_t cap = 3 * k + 16384;
+        if (cap > d) cap = d;
+        c->cand_cap = uint32_t(cap);
+    }
+
+    // carve the workspace; the first region (histograms, counters) is what reset() clears
+    size_t off = 0;
+    auto carve = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t o_samp = carve(NCOARSE * 4), o_cw = carve((WIN + 1) * 4), o_ctrl = carve(CT_WORDS * 4), o_bar = carve(8);
+    const size_t o_bt = carve(size_t(c->topk_blocks) * 4);
+    c->ctrl_region_bytes = off;
+    const size_t o_fine = carve(NFINE * 4), o_dh = carve(size_t(DH_PASSES) * DH_BINS * 4);
+    const size_t o_cand = carve(size_t(c->cand_cap) * 8);
+    const size_t o_bm = carve(size_t(c->ntiles) * 32 * 4), o_tp = carve((size_t(c->ntiles) + 1) * 4);
+    c->ws_bytes = off;
+    if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return SCALECOM_ERR_ALLOC;
+    }
+    char* base = static_cast<char*>(c->ws);
+    c->samp_hist = reinterpret_cast<uint32_t*>(base + o_samp);
+    c->coarse_win = reinterpret_cast<uint32_t*>(base + o_cw);
+    c->ctrl = reinterpret_cast<uint32_t*>(base + o_ctrl);
+    c->barrier = reinterpret_cast<unsigned long long*>(base + o_bar);
+    c->block_tot = reinterpret_cast<uint32_t*>(base + o_bt);
+    c->fine_hist = reinterpret_cast<uint32_t*>(base + o_fine);
+    c->digit_hist = reinterpret_cast<uint32_t*>(base + o_dh);
+    c->cand = reinterpret_cast<uint2*>(base + o_cand);
+    c->bitmap = reinterpret_cast<uint32_t*>(base + o_bm);
+    c->tile_prefix = reinterpret_cast<uint32_t*>(base + o_tp);
+
+    bool ok = init_workspace(c) == SCALECOM_OK;
+    for (int i = 0; ok && i < 4; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) {
+        cudaGetLastError();
+        scalecom_destroy(c);
+        return SCALECOM_ERR_CUDA;
+    }
+    *out = c;
+    return SCALECOM_OK;
+}
+
+int scalecom_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float* weights, int64_t t,
+                  int32_t* out_idx, float* out_val) {
+    const int rc = check_step_args(c, reinterpret_cast<const void* const*>(grads),
+                                   reinterpret_cast<const void* const*>(mem), weights, t, out_idx, out_val);
+    if (rc != SCALECOM_OK) return rc;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    return do_step(c, grads, mem, weights, t, out_idx, out_val);
+}
+
+int scalecom_step_host(scalecom_ctx* c, const float* const* host_grads, float* const* mem, float* weights, int64_t t,
+                       int32_t* host_idx, float* host_val) {
+    if (!c || !host_grads || !mem || !host_idx || !host_val) return SCALECOM_ERR_NULL_PTR;
+    if (t < 0) return SCALECOM_ERR_INVALID_ARG;
+    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
+    for (int i = 0; i < c->n; ++i)
+        if (!host_grads[i] || !mem[i]) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    if (!c->stage_g) {
+        const size_t gbytes = size_t(c->n) * size_t(c->d) * 4;
+        if (cudaMalloc(reinterpret_cast<void**>(&c->stage_g), gbytes) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&c->stage_idx), size_t(c->k) * 4) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&c->stage_val), size_t(c->k) * 4) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(c->stage_g); cudaFree(c->stage_idx); cudaFree(c->stage_val);
+            c->stage_g = nullptr; c->stage_idx = nullptr; c->stage_val = nullptr;
+            return SCALECOM_ERR_ALLOC;
+        }
+    }
+    const float* dev_g[SCALECOM_MAX_LEARNERS];
+    const int leader = int(t % c->n);
+    // the leader's gradient goes first: the selection kernel needs nothing else
+    for (int j = 0; j < c->n; ++j) {
+        const int i = (leader + j) % c->n;
+        float* dst = c->stage_g + size_t(i) * size_t(c->d);
+        dev_g[i] = dst;
+        if (cudaMemcpyAsync(dst, host_grads[i], size_t(c->d) * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+            return SCALECOM_ERR_CUDA;
+    }
+    int rc = check_step_args(c, reinterpret_cast<const void* const*>(dev_g), reinterpret_cast<const void* const*>(mem),
+                             weights, t, c->stage_idx, c->stage_val);
+    if (rc != SCALECOM_OK) return rc;
+    rc = do_step(c, dev_g, mem, weights, t, c->stage_idx, c->stage_val);
+    if (rc != SCALECOM_OK) return rc;
+    if (cudaMemcpyAsync(host_idx, c->stage_idx, size_t(c->k) * 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaMemcpyAsync(host_val, c->stage_val, size_t(c->k) * 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+        return SCALECOM_ERR_CUDA;
+    return SCALECOM_OK;
+}
+
+void scalecom_destroy(scalecom_ctx* c) {
+    if (!c) return;
+    DeviceGuard guard(c->device);
+    cudaStreamSynchronize(c->stream);
+    for (auto& e : c->ev)
+        if (e) cudaEventDestroy(e);
+    cudaFree(c->ws);
+    cudaFree(c->stage_g);
+    cudaFree(c->stage_idx);
+    cudaFree(c->stage_val);
+    cudaGetLastError();
+    delete c;
+}
+
+int scalecom_set_stream(scalecom_ctx* c, void* cuda_stream) {
+    if (!c) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;   // scratch is shared between steps
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    return SCALECOM_OK;
+}
+
+int scalecom_set_gathered(scalecom_ctx* c, float* dev_gathered) {
+    if (!c) return SCALECOM_ERR_NULL_PTR;
+    c->gathered = dev_gathered;
+    return SCALECOM_OK;
+}
+
+int scalecom_apply_update(scalecom_ctx* c, float* weights, const int32_t* idx, const float* val, int64_t k, float lr) {
+    if (!c || !weights || !idx || !val) return SCALECOM_ERR_NULL_PTR;
+    if (k < 0 || k > c->d || !std::isfinite(lr)) return SCALECOM_ERR_INVALID_ARG;
+    if (k == 0) return SCALECOM_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    const uint32_t blocks = uint32_t((k + 255) / 256);
+    apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, idx, val, uint32_t(k), lr);
+    if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+    ++c->launches;
+    return SCALECOM_OK;
+}
+
+int scalecom_status(scalecom_ctx* c) {
+    if (!c) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    uint32_t st = 0;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
+        cudaMemcpy(&st, c->ctrl + CT_STATUS, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        c->poisoned = true;
+        return SCALECOM_ERR_CUDA;
+    }
+    if (st == DEV_OK) return SCALECOM_OK;
+    c->poisoned = true;
+    return st == DEV_TIMEOUT ? SCALECOM_ERR_TIMEOUT : SCALECOM_ERR_INTERNAL;
+}
+
+int scalecom_reset(scalecom_ctx* c) {
+    if (!c) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (init_workspace(c) != SCALECOM_OK || cudaStreamSynchronize(c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    c->poisoned = false;
+    return SCALECOM_OK;
+}
+
+int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
+    if (!c) return SCALECOM_ERR_NULL_PTR;
+    switch (option) {
+        case SCALECOM_OPT_FORCE_EXACT_PATH: c->force_exact = value ? 1u : 0u; return SCALECOM_OK;
+        case SCALECOM_OPT_SPIN_LIMIT:
+            if (value < 0 || value > 0x7FFFFFFFLL) return SCALECOM_ERR_INVALID_ARG;
+            c->spin_limit = uint32_t(value);
+            return SCALECOM_OK;
+        case SCALECOM_OPT_KERNEL_TIMING: c->timing = value != 0; c->ev_valid = false; return SCALECOM_OK;
+        case SCALECOM_OPT_FUSE_UPDATE: c->fuse_update = value != 0; return SCALECOM_OK;
+        default: return SCALECOM_ERR_INVALID_ARG;
+    }
+}
+
+int scalecom_query(scalecom_ctx* c, int item, int64_t* out) {
+    if (!c || !out) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    uint32_t w[CT_WORDS];
+    switch (item) {
+        case SCALECOM_Q_WORKSPACE_BYTES:
+            *out = int64_t(c->ws_bytes) + (c->stage_g ? int64_t(c->n) * c->d * 4 + c->k * 8 : 0);
+            return SCALECOM_OK;
+        case SCALECOM_Q_TOPK_BLOCKS: *out = c->topk_blocks; return SCALECOM_OK;
+        case SCALECOM_Q_KERNEL_LAUNCHES: *out = c->launches; return SCALECOM_OK;
+        case SCALECOM_Q_LAST_TOPK_PATH:
+        case SCALECOM_Q_LAST_CANDIDATES:
+            if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
+                cudaMemcpy(w, c->ctrl, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess)
+                return SCALECOM_ERR_CUDA;
+            *out = item == SCALECOM_Q_LAST_TOPK_PATH ? w[CT_PATH] : w[CT_M];
+            return SCALECOM_OK;
+        default: return SCALECOM_ERR_INVALID_ARG;
+    }
+}
+
+int scalecom_last_kernel_ms(scalecom_ctx* c, float ms[3]) {
+    if (!c || !ms) return SCALECOM_ERR_NULL_PTR;
+    if (!c->timing || !c->ev_valid) return SCALECOM_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (cudaEventSynchronize(c->ev[3]) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    for (int i = 0; i < 3; ++i)
+        if (cudaEventElapsedTime(&ms[i], c->ev[i], c->ev[i + 1]) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    return SCALECOM_OK;
+}
+
+const char* scalecom_strerror(int code) {
+    switch (code) {
+        case SCALECOM_OK: return "success";
+        case SCALECOM_ERR_INVALID_ARG: return "invalid argument";
+        case SCALECOM_ERR_NULL_PTR: return "null pointer";
+        case SCALECOM_ERR_ALLOC: return "allocation failed";
+        case SCALECOM_ERR_CUDA: return "CUDA runtime error";
+        case SCALECOM_ERR_TIMEOUT: return "device-side wait timed out";
+        case SCALECOM_ERR_BAD_STATE: return "handle in error state (call scalecom_reset)";
+        case SCALECOM_ERR_INTERNAL: return "device-side consistency check failed";
+        case SCALECOM_ERR_ALIAS: return "buffers overlap";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

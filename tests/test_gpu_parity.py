@@ -1,0 +1,153 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2104_11125_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _parity():
+    from tests import parity
+    return parity
+
+
+def _t(a):
+    return torch.tensor(np.asarray(a, np.float32), device=DEV)
+
+
+# ---- the paper-shaped workloads at sizes the oracle finishes in seconds ---------------------------
+@pytest.mark.parametrize("force_exact", [False, True])
+def test_tiny_config_full(force_exact):
+    """Config 1 exactly as specified: n=4, d=2^20, k=d/100, 10 steps, leader t mod 4."""
+    _parity().workload_case(W.TINY, W.TINY.steps if not force_exact else 3, DEV, force_exact=force_exact,
+                            want_path=1 if force_exact else 0)
+
+
+@pytest.mark.parametrize("base,d,n,steps", [
+    (W.RESNET50, 1_500_013, 8, 4),          # several tiles of every kernel plus a ragged tail (d odd)
+    (W.TRANSFORMER, 2_000_003, 16, 3),
+    (W.LARGE, 3_000_001, 5, 3),
+    (W.RESNET50, 300_007, 20, 3),           # > 16 learners: second pointer-table size
+    (W.RESNET50, 50_001, 130, 2),           # > 128 learners: third pointer-table size
+])
+def test_scaled_workloads(base, d, n, steps):
+    _parity().workload_case(base.scaled(d, n=n), steps, DEV, want_path=0)
+
+
+def test_separate_update_kernel_and_no_weights():
+    w = W.TINY.scaled(200_000)
+    _parity().workload_case(w, 3, DEV, fuse_update=False)
+    p = _parity()
+    prof = W.profile(w, DEV)
+    grads = [W.gradients(w, s, DEV, prof) for s in range(2)]
+    p.run_and_compare(grads, W.initial_memory(w, DEV), None, w.k, w.beta, w.lr, tag="no-weights")
+
+
+@pytest.mark.parametrize("offset", [1, 2, 3])
+def test_unaligned_vectors(offset):
+    w = W.TINY.scaled(100_003)
+    _parity().workload_case(w, 2, DEV, offset=offset)
+    _parity().workload_case(w, 2, DEV, offset=offset, force_exact=True)
+
+
+# ---- edge cases -------------------------------------------------------------------------------------
+def _edge(g_rows, k, beta=0.5, lr=0.25, steps=3, m_rows=None, **kw):
+    g = [_t(r) for r in g_rows]
+    n, d = len(g), g[0].numel()
+    m0 = [_t(r) for r in m_rows] if m_rows is not None else [torch.zeros(d, device=DEV) for _ in range(n)]
+    theta = torch.linspace(-1, 1, d, device=DEV)
+    return _parity().run_and_compare([g] * steps, m0, theta, k, beta, lr, **kw)
+
+
+@pytest.mark.parametrize("force_exact", [False, True])
+def test_degenerate_inputs(force_exact):
+    rng = np.random.default_rng(5)
+    kw = dict(force_exact=force_exact)
+    _edge([[3.0]], 1, tag="d=1", **kw)
+    _edge([[0.0, 0.0, 0.0, 0.0, 0.0]] * 2, 2, tag="all-zero", **kw)
+    _edge([np.zeros(5000)] * 3, 77, tag="all-zero-5000", **kw)
+    _edge([np.full(4099, 2.5), np.full(4099, -2.5)], 100, tag="all-equal", **kw)
+    pm = np.where(np.arange(9001) % 2 == 0, 1.0, -1.0)
+    _edge([pm, -pm, pm], 4500, tag="plus-minus-ties", **kw)
+    x = rng.standard_normal(10_000)
+    _edge([x, x * 0.5], 1, tag="k=1", **kw)
+    _edge([x, x * 0.5], 10_000, tag="k=d", **kw)
+    _edge([x], 100, beta=1.0, tag="n=1,beta=1", **kw)
+    den = (rng.integers(-5, 6, 7001) * 1e-41).astype(np.float32)
+    _edge([den, den[::-1].copy()], 300, tag="denormals", **kw)
+    q = rng.integers(-3, 4, 50_000).astype(np.float32)          # heavy ties at every level
+    _edge([q, np.roll(q, 1)], 5000, tag="quantised", **kw)
+    neg0 = np.array([-0.0, 0.0, -0.0, 1.0, -1.0, 0.0, -0.0], np.float32)
+    _edge([neg0, -neg0], 3, tag="signed-zeros", **kw)
+
+
+def test_ties_straddling_rank_k_on_the_fast_path():
+    """Equal magnitudes on both sides of rank k with the candidate list in use:
+    the winners among equals must be the lowest indices."""
+    rng = np.random.default_rng(9)
+    d, k = 400_000, 4000
+    x = rng.standard_normal(d).astype(np.float32)
+    order = np.argsort(-np.abs(x))
+    tau = abs(x[order[k - 1]])
+    ties = rng.choice(d, 600, replace=False)
+    x[ties] = np.where(rng.random(600) < 0.5, tau, -tau)        # ~600 copies of the k-th magnitude
+    paths = _edge([x, 0.9 * x, 1.1 * x], k, steps=3, tag="ties-at-k")
+    assert paths[0] == 0
+
+
+def test_many_learners_small_vector():
+    w = W.RESNET50.scaled(20_011, n=128)
+    _parity().workload_case(w, 2, DEV)
+
+
+def test_resume_equals_uninterrupted_run():
+    """All state is the caller's: 4 steps with one handle == 2 + 2 steps with two handles."""
+    import paper_2104_11125_b200 as sc
+    w = W.TINY.scaled(150_001)
+    prof = W.profile(w, DEV)
+    grads = [W.gradients(w, s, DEV, prof) for s in range(4)]
+
+    def run(split):
+        m = W.initial_memory(w, DEV)
+        th = W.initial_weights(w, DEV)
+        idx = torch.empty(w.k, device=DEV, dtype=torch.int32)
+        val = torch.empty(w.k, device=DEV)
+        outs = []
+        for lo, hi in split:
+            with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
+                for t in range(lo, hi):
+                    ctx.step(grads[t], m, th, t, idx, val)
+                    outs.append((idx.clone(), val.clone()))
+                assert ctx.status() == 0
+        return m, th, outs
+
+    m1, th1, o1 = run([(0, 4)])
+    m2, th2, o2 = run([(0, 2), (2, 4)])
+    assert all(torch.equal(a, b) for a, b in zip(m1, m2)) and torch.equal(th1, th2)
+    assert all(torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]) for a, b in zip(o1, o2))
+
+
+def test_host_buffer_entry_point():
+    import paper_2104_11125_b200 as sc
+    import oracle
+    w = W.TINY.scaled(120_000)
+    prof = W.profile(w, DEV)
+    m = W.initial_memory(w, DEV)
+    th = W.initial_weights(w, DEV)
+    m_o = [x.cpu().numpy().copy() for x in m]
+    th_o = th.cpu().numpy().copy()
+    hidx = torch.empty(w.k, dtype=torch.int32).pin_memory()
+    hval = torch.empty(w.k, dtype=torch.float32).pin_memory()
+    with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
+        for t in range(3):
+            hg = [g.cpu().pin_memory() for g in W.gradients(w, t, DEV, prof)]
+            ctx.step_host(hg, m, th, t, hidx, hval)
+            idx_o, val_o, _ = oracle.step([g.numpy() for g in hg], m_o, th_o, t, w.k, w.beta, w.lr)
+            assert np.array_equal(hidx.numpy(), idx_o) and np.array_equal(hval.numpy(), val_o)
+        assert ctx.status() == 0
+    assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(m, m_o))
+    assert np.array_equal(th.cpu().numpy(), th_o)
