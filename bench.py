@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the CLT-k step: learner-elements/s (n*d / step time) and HBM roofline fraction.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50] [--impl reference]
+
+One "step" is one scalecom_step call (selection on the leader, fused learner
+pass over all n learners, weight update) on seeded synthetic gradients of the
+named workload.  N > 1 (under torchrun) runs N independent replicas: the
+method keeps all n logical learners inside one GPU, so nothing is exchanged.
+Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "learner-elements/s per CLT-k step (n*d/step time)"
+UNIT = "learner-elements/s"
+FALLBACK_HBM_GBS = 6650.0            # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+NOMINAL_HBM_GBS = 8000.0
+MAX_BATCHES = 24                     # distinct gradient batches kept resident; steps cycle through them
+
+# DRAM traffic per launch of the learner pass on the bench workload from an ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum); None until captured.
+NCU_TRAFFIC_BYTES = {"resnet50": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def get_workload(name):
+    from paper_2104_11125_b200 import workloads as W
+    if name in W.CONFIGS:
+        return W.CONFIGS[name]
+    if name.startswith("resnet50_n"):
+        return W.sweep(int(name[len("resnet50_n"):]))
+    raise SystemExit("unknown workload %r (have %s, resnet50_n<N>)" % (name, ", ".join(W.CONFIGS)))
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, device_index):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # pragma: no cover
+            self.error = repr(e)
+
+    def run(self):
+        if self._h is None:
+            return
+        nv = self._nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.001)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def cpu_threads():
+    return 1          # the oracle is plain single-threaded C
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, timed on host cores on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2104_11125_b200 import workloads as W
+    full = get_workload(args.workload)
+    d_s = min(full.d, 2_000_000)
+    w = full.scaled(d_s)
+    prof = W.profile(w, "cpu")
+    nb = min(args.steps + args.warmup, 4)
+    batches = [[g.numpy() for g in W.gradients(w, s, "cpu", prof)] for s in range(nb)]
+    m = [x.numpy() for x in W.initial_memory(w, "cpu")]
+    th = W.initial_weights(w, "cpu").numpy()
+    t = 0
+    for _ in range(args.warmup):
+        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False)
+        t += 1
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False)
+        t += 1
+    dt = time.perf_counter() - t0
+    value = w.n * w.d * args.steps / dt
+    sample = "first %d of %d coordinates per learner (same recipe, n=%d, k=%d), every step" % (w.d, full.d, w.n, w.k)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": full.name, "n": full.n, "d": full.d, "k": full.k, "beta": full.beta, "lr": full.lr,
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def time_oracle(w, batches_dev, steps=2):
+    """cpu_baseline leg: the oracle on full-size steps of the bench workload, on this machine's host cores."""
+    import numpy as np
+    import oracle
+    m = [np.zeros(w.d, np.float32) for _ in range(w.n)]
+    th = np.zeros(w.d, np.float32)
+    dt = 0.0
+    for s in range(steps):
+        g = [x.cpu().numpy() for x in batches_dev[s % len(batches_dev)]]
+        t0 = time.perf_counter()
+        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False)
+        dt += time.perf_counter() - t0
+    return {"value": w.n * w.d * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+            "sample": "%d full steps of the bench workload (n=%d, d=%d, k=%d), %.1f s" % (steps, w.n, w.d, w.k, dt)}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding, workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = get_workload(args.workload)
+    K, Wm = args.steps, max(args.warmup, 3)
+    prof = W.profile(w, dev)
+    nb = min(K + Wm, MAX_BATCHES)
+    batches = [W.gradients(w, s, dev, prof) for s in range(nb)]
+    mem = W.initial_memory(w, dev)
+    theta = W.initial_weights(w, dev)
+    idx = torch.empty(w.k, device=dev, dtype=torch.int32)
+    val = torch.empty(w.k, device=dev, dtype=torch.float32)
+
+    stream = torch.cuda.Stream(device=dev)
+    ctx = sc.Context(w.d, w.n, w.k, w.beta, w.lr, stream=stream)
+    ctx.set_option(binding.OPT_KERNEL_TIMING, 1)
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing ---------------------------------------------------------------------
+    t = 0
+    for _ in range(Wm):
+        ctx.step(batches[t % nb], mem, theta, t, idx, val)
+        t += 1
+    ctx.kernel_ms()                                   # drop the warm-up records
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.query(binding.Q_KERNEL_LAUNCHES)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev0.record(stream)
+    for _ in range(K):
+        ctx.step(batches[t % nb], mem, theta, t, idx, val)
+        t += 1
+    ev1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = ctx.query(binding.Q_KERNEL_LAUNCHES) - launches0
+    assert ctx.status() == 0, "device status %d" % ctx.status()
+    kms, ksteps = ctx.kernel_ms()
+    paths = ctx.query(binding.Q_LAST_TOPK_PATH)
+
+    # ---- end to end through the host-buffer entry point ------------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        hb = [[g.cpu().pin_memory() for g in batches[s]] for s in range(min(2, nb))]
+        hidx = torch.empty(w.k, dtype=torch.int32).pin_memory()
+        hval = torch.empty(w.k, dtype=torch.float32).pin_memory()
+        ke = max(3, min(K, 20))
+        for s in range(2):
+            ctx.step_host(hb[s % len(hb)], mem, theta, t, hidx, hval)
+            t += 1
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for s in range(ke):
+            ctx.step_host(hb[s % len(hb)], mem, theta, t, hidx, hval)
+            t += 1
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / ke
+        del hb
+    else:
+        e2e_ms = None
+
+    # ---- max over ranks --------------------------------------------------------------------------------
+    if world > 1:
+        tt = torch.tensor([ms_total, e2e_ms or 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total, e2e_max = float(tt[0]), float(tt[1])
+        e2e_ms = e2e_max if e2e_ms is not None else None
+
+    if rank == 0:
+        ms_step = ms_total / K
+        units = w.n * w.d * world
+        peak, peak_src = measured_peak()
+        lp_ms = kms[1] / max(ksteps, 1)
+        tk_ms = kms[0] / max(ksteps, 1)
+        lp_bytes = 12.0 * w.n * w.d
+        tk_bytes = 8.0 * w.d + 4.0 * w.k
+        lp_gbs = lp_bytes / (lp_ms * 1e-3) / 1e9
+        tk_gbs = tk_bytes / (tk_ms * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": units / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "n": w.n, "d": w.d, "k": w.k, "beta": w.beta, "lr": w.lr,
+                       "parallelism": "replicas only" if world > 1 else "single GPU, n logical learners",
+                       "l2": "inputs larger than L2 (%.2f GB of g+m per step), no flush" % (8e-9 * w.n * w.d),
+                       "gradient_batches_resident": nb, "selection_path_last_step": paths,
+                       "weight_update": "fused into the learner pass"},
+            "roofline": {"bound": "hbm", "kernel": "learner_pass_kernel", "achieved": lp_gbs, "peak": peak,
+                         "unit": "GB/s", "frac": lp_gbs / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": lp_bytes, "avg_launch_ms": lp_ms,
+                         "frac_of_nominal_8TBs": lp_gbs / NOMINAL_HBM_GBS,
+                         "topk_select_kernel": {"achieved": tk_gbs, "frac": tk_gbs / peak, "avg_launch_ms": tk_ms,
+                                                "algorithmic_bytes_per_launch": tk_bytes,
+                                                "frac_of_nominal_8TBs": tk_gbs / NOMINAL_HBM_GBS},
+                         "steps_timed": ksteps},
+            "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        if e2e_ms is not None:
+            out["e2e"] = {"value": units / (e2e_ms * 1e-3), "unit": UNIT,
+                          "h2d_bytes_per_step": 4 * w.n * w.d, "d2h_bytes_per_step": 8 * w.k,
+                          "ms_per_step": e2e_ms, "api": "scalecom_step_host (pinned host gradients in, idx/val out)"}
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = time_oracle(w, batches)
+        print(json.dumps(out))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -156,11 +156,15 @@ int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 int scalecom_query(scalecom_ctx* ctx, int item, int64_t* out);
 
 /*
- * With SCALECOM_OPT_KERNEL_TIMING on: waits for the last step and writes its
- * kernel durations in milliseconds: ms[0] selection (step 2), ms[1] learner
- * pass (steps 1, 3, 4, and 5 when fused), ms[2] separate weight update (0 when fused).
+ * With SCALECOM_OPT_KERNEL_TIMING on, every step brackets its kernels with CUDA
+ * events on the handle's stream (the most recent 256 steps are kept).  This call
+ * waits for the stream, writes the durations in milliseconds SUMMED over the
+ * steps recorded since the previous call (or since timing was switched on) and
+ * forgets them: ms[0] selection (step 2), ms[1] learner pass (steps 1, 3, 4, and
+ * 5 when fused), ms[2] separate weight update (0 when fused); *nsteps receives
+ * the number of steps summed.  BAD_STATE when timing is off.
  */
-int scalecom_last_kernel_ms(scalecom_ctx* ctx, float ms[3]);
+int scalecom_kernel_ms(scalecom_ctx* ctx, float ms[3], int32_t* nsteps);
 
 /* Static, never NULL. */
 const char* scalecom_strerror(int code);

@@ -27,7 +27,7 @@ Q_WORKSPACE_BYTES, Q_LAST_TOPK_PATH, Q_LAST_CANDIDATES, Q_TOPK_BLOCKS, Q_KERNEL_
 EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
-    "scalecom_set_option", "scalecom_query", "scalecom_last_kernel_ms", "scalecom_strerror",
+    "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
 )
 
 _lib = None
@@ -71,8 +71,8 @@ def lib() -> ctypes.CDLL:
         L.scalecom_set_option.argtypes = [vp, ctypes.c_int, i64]
         L.scalecom_query.restype = ctypes.c_int
         L.scalecom_query.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64)]
-        L.scalecom_last_kernel_ms.restype = ctypes.c_int
-        L.scalecom_last_kernel_ms.argtypes = [vp, ctypes.POINTER(f32)]
+        L.scalecom_kernel_ms.restype = ctypes.c_int
+        L.scalecom_kernel_ms.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(i32)]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -173,10 +173,12 @@ class Context:
     def reset(self) -> None:
         _check(lib().scalecom_reset(self._h), "scalecom_reset")
 
-    def last_kernel_ms(self) -> List[float]:
+    def kernel_ms(self) -> Tuple[List[float], int]:
+        """(summed kernel milliseconds [selection, learner pass, separate update], steps summed)."""
         ms = (ctypes.c_float * 3)()
-        _check(lib().scalecom_last_kernel_ms(self._h, ms), "scalecom_last_kernel_ms")
-        return list(ms)
+        ns = ctypes.c_int32()
+        _check(lib().scalecom_kernel_ms(self._h, ms, ctypes.byref(ns)), "scalecom_kernel_ms")
+        return list(ms), ns.value
 
     def step(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], weights: Optional[torch.Tensor],
              t: int, out_idx: torch.Tensor, out_val: torch.Tensor) -> None:

@@ -48,8 +48,10 @@ struct scalecom_ctx {
     int32_t* stage_idx = nullptr;      // k
     float* stage_val = nullptr;        // k
 
-    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
-    bool ev_valid = false;
+    // kernel timing: a ring of 4 events per step
+    static constexpr int EV_RING = 256;
+    cudaEvent_t* ev = nullptr;         // [EV_RING * 4], created when timing is first switched on
+    int64_t ev_steps = 0;              // steps recorded since the last read
     bool poisoned = false;
     int64_t launches = 0;
 };
@@ -173,16 +175,17 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     for (int i = 0; i < c->n; ++i) vec_all = vec_all && aligned16(grads[i]) && aligned16(mem[i]);
     const bool vec_leader = aligned16(tp.g) && aligned16(tp.m);
 
-    const bool tm = c->timing;
-    if (tm && cudaEventRecord(c->ev[0], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    const bool tm = c->timing && c->ev;
+    cudaEvent_t* ev = tm ? c->ev + 4 * (c->ev_steps % scalecom_ctx::EV_RING) : nullptr;
+    if (tm && cudaEventRecord(ev[0], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     cudaError_t e = vec_leader ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
-    if (tm && cudaEventRecord(c->ev[1], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (tm && cudaEventRecord(ev[1], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     e = vec_all ? launch_learner_n<true>(c, grads, mem, lp) : launch_learner_n<false>(c, grads, mem, lp);
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
-    if (tm && cudaEventRecord(c->ev[2], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (tm && cudaEventRecord(ev[2], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     if (weights && !c->fuse_update) {
         const uint32_t blocks = uint32_t((c->k + 255) / 256);
         apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, out_idx, out_val,
@@ -191,8 +194,8 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
         ++c->launches;
     }
     if (tm) {
-        if (cudaEventRecord(c->ev[3], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
-        c->ev_valid = true;
+        if (cudaEventRecord(ev[3], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+        ++c->ev_steps;
     }
     return SCALECOM_OK;
 }
@@ -295,8 +298,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->bitmap = reinterpret_cast<uint32_t*>(base + o_bm);
     c->tile_prefix = reinterpret_cast<uint32_t*>(base + o_tp);
 
-    bool ok = init_workspace(c) == SCALECOM_OK;
-    for (int i = 0; ok && i < 4; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    const bool ok = init_workspace(c) == SCALECOM_OK;
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) {
         cudaGetLastError();
         scalecom_destroy(c);
@@ -362,8 +364,11 @@ void scalecom_destroy(scalecom_ctx* c) {
     if (!c) return;
     DeviceGuard guard(c->device);
     cudaStreamSynchronize(c->stream);
-    for (auto& e : c->ev)
-        if (e) cudaEventDestroy(e);
+    if (c->ev) {
+        for (int i = 0; i < scalecom_ctx::EV_RING * 4; ++i)
+            if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+        delete[] c->ev;
+    }
     cudaFree(c->ws);
     cudaFree(c->stage_g);
     cudaFree(c->stage_idx);
@@ -430,7 +435,18 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
             if (value < 0 || value > 0x7FFFFFFFLL) return SCALECOM_ERR_INVALID_ARG;
             c->spin_limit = uint32_t(value);
             return SCALECOM_OK;
-        case SCALECOM_OPT_KERNEL_TIMING: c->timing = value != 0; c->ev_valid = false; return SCALECOM_OK;
+        case SCALECOM_OPT_KERNEL_TIMING: {
+            if (value && !c->ev) {
+                DeviceGuard guard(c->device);
+                c->ev = new (std::nothrow) cudaEvent_t[scalecom_ctx::EV_RING * 4]();
+                if (!c->ev) return SCALECOM_ERR_ALLOC;
+                for (int i = 0; i < scalecom_ctx::EV_RING * 4; ++i)
+                    if (cudaEventCreate(&c->ev[i]) != cudaSuccess) return SCALECOM_ERR_CUDA;
+            }
+            c->timing = value != 0;
+            c->ev_steps = 0;
+            return SCALECOM_OK;
+        }
         case SCALECOM_OPT_FUSE_UPDATE: c->fuse_update = value != 0; return SCALECOM_OK;
         default: return SCALECOM_ERR_INVALID_ARG;
     }
@@ -457,13 +473,23 @@ int scalecom_query(scalecom_ctx* c, int item, int64_t* out) {
     }
 }
 
-int scalecom_last_kernel_ms(scalecom_ctx* c, float ms[3]) {
-    if (!c || !ms) return SCALECOM_ERR_NULL_PTR;
-    if (!c->timing || !c->ev_valid) return SCALECOM_ERR_BAD_STATE;
+int scalecom_kernel_ms(scalecom_ctx* c, float ms[3], int32_t* nsteps) {
+    if (!c || !ms || !nsteps) return SCALECOM_ERR_NULL_PTR;
+    if (!c->timing || !c->ev) return SCALECOM_ERR_BAD_STATE;
     DeviceGuard guard(c->device);
-    if (cudaEventSynchronize(c->ev[3]) != cudaSuccess) return SCALECOM_ERR_CUDA;
-    for (int i = 0; i < 3; ++i)
-        if (cudaEventElapsedTime(&ms[i], c->ev[i], c->ev[i + 1]) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    const int64_t kept = c->ev_steps < scalecom_ctx::EV_RING ? c->ev_steps : scalecom_ctx::EV_RING;
+    ms[0] = ms[1] = ms[2] = 0.f;
+    for (int64_t s = c->ev_steps - kept; s < c->ev_steps; ++s) {
+        cudaEvent_t* ev = c->ev + 4 * (s % scalecom_ctx::EV_RING);
+        for (int i = 0; i < 3; ++i) {
+            float x = 0.f;
+            if (cudaEventElapsedTime(&x, ev[i], ev[i + 1]) != cudaSuccess) return SCALECOM_ERR_CUDA;
+            ms[i] += x;
+        }
+    }
+    *nsteps = int32_t(kept);
+    c->ev_steps = 0;
     return SCALECOM_OK;
 }
 

@@ -103,8 +103,9 @@ def segments(w: Workload) -> List[Tuple[int, int]]:
         return [(0, w.d)]
     total = sum(base)
     sizes = [max(1, (s * w.d) // total) for s in base] if total != w.d else list(base)
-    sizes[-1] += w.d - sum(sizes)
-    if sizes[-1] < 1:
+    big = max(range(len(sizes)), key=lambda i: sizes[i])      # rounding slack goes to the largest segment
+    sizes[big] += w.d - sum(sizes)
+    if sizes[big] < 1:
         raise ValueError("d too small for the segment layout")
     out, off = [], 0
     for s in sizes:
