@@ -153,6 +153,8 @@ int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */
+#define SCALECOM_Q_PHASE_STAMP0     100 /* +i, i < 10: low 32 bits of the GPU nanosecond timer when block 0 of
+                                          the last selection kernel reached phase boundary i (profiling aid)   */
 int scalecom_query(scalecom_ctx* ctx, int item, int64_t* out);
 
 /*

@@ -469,7 +469,15 @@ int scalecom_query(scalecom_ctx* c, int item, int64_t* out) {
                 return SCALECOM_ERR_CUDA;
             *out = item == SCALECOM_Q_LAST_TOPK_PATH ? w[CT_PATH] : w[CT_M];
             return SCALECOM_OK;
-        default: return SCALECOM_ERR_INVALID_ARG;
+        default:
+            if (item >= SCALECOM_Q_PHASE_STAMP0 && item < SCALECOM_Q_PHASE_STAMP0 + CT_NSTAMPS) {
+                if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
+                    cudaMemcpy(w, c->ctrl, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess)
+                    return SCALECOM_ERR_CUDA;
+                *out = w[CT_STAMP + item - SCALECOM_Q_PHASE_STAMP0];
+                return SCALECOM_OK;
+            }
+            return SCALECOM_ERR_INVALID_ARG;
     }
 }
 

@@ -42,7 +42,7 @@ constexpr uint32_t WCAP = 192;                                 // candidate stag
 constexpr uint32_t SAMPLE_GRANULE = 128;                       // coordinates one warp samples at a time
 
 // ctrl words
-constexpr int CT_CAND = 0, CT_STATUS = 1, CT_PATH = 2, CT_M = 3, CT_WORDS = 8;
+constexpr int CT_CAND = 0, CT_STATUS = 1, CT_PATH = 2, CT_M = 3, CT_STAMP = 8, CT_NSTAMPS = 10, CT_WORDS = 32;
 
 struct TopkParams {
     const float* g;            // leader's gradient, fp32[d]
@@ -71,49 +71,66 @@ struct TopkParams {
 struct TopkShared {
     uint32_t hist[NCOARSE];            // sample histogram / staging for bin searches / digit histogram
     uint2 stage[TK_WARPS][WCAP];       // per-warp candidate staging
+    uint32_t cw[WIN + 1];              // this block's share of the coarse window histogram
     uint32_t scan[32];
     uint32_t res[4];
     int flag;
 };
 
-// Search a histogram from its top bin downwards for the bin holding the
-// `need`-th element: res = {bin, count strictly above bin, count in bin}, or
-// bin = 0xFFFFFFFF when the histogram holds fewer than `need` elements.
+// Search a histogram (global memory, written by other blocks before the last
+// grid barrier) from its top bin downwards for the bin holding the `need`-th
+// element: res = {bin, count strictly above bin, count in bin}, or bin =
+// 0xFFFFFFFF when the histogram holds fewer than `need` elements.  nb <= 8192.
+// Two levels, both with one bin per lane per load (coalesced, no bank
+// conflicts): 16 warp-sized segments, then 16 sub-segments of <= 32 bins.
 __device__ inline void find_from_top(const uint32_t* h, uint32_t nb, uint32_t need, TopkShared& s) {
-    const uint32_t tid = threadIdx.x;
-    if (tid == 0) s.res[0] = 0xFFFFFFFFu;
-    const uint32_t chunk = (nb + TK_THREADS - 1) / TK_THREADS;
-    const uint32_t r0 = tid * chunk;
-    uint32_t sum = 0;
-    for (uint32_t j = 0; j < chunk; ++j) {
-        const uint32_t r = r0 + j;
-        if (r < nb) sum += h[nb - 1 - r];
-    }
-    const uint32_t incl = warp_incl_scan(sum);
-    if (lane_id() == 31) s.scan[warp_id()] = incl;
-    __syncthreads();
-    if (warp_id() == 0) {
-        const uint32_t v = lane_id() < TK_WARPS ? s.scan[lane_id()] : 0u;
-        const uint32_t vi = warp_incl_scan(v);
-        s.scan[lane_id()] = vi - v;
+    const uint32_t lane = lane_id(), warp = warp_id();
+    if (threadIdx.x == 0) s.res[0] = 0xFFFFFFFFu;
+    // level 1: warp w sums reversed positions [w*seglen, (w+1)*seglen)
+    const uint32_t seglen = (nb + TK_WARPS - 1) / TK_WARPS;
+    {
+        const uint32_t r0 = warp * seglen, r1 = min(nb, r0 + seglen);
+        uint32_t sum = 0;
+        for (uint32_t r = r0 + lane; r < r1; r += 32) sum += __ldcg(h + (nb - 1 - r));
+        sum = warp_sum(sum);
+        if (lane == 0) s.scan[warp] = sum;
     }
     __syncthreads();
-    const uint32_t excl = s.scan[warp_id()] + incl - sum;
-    if (excl < need && need <= excl + sum) {
-        uint32_t run = excl;
-        for (uint32_t j = 0; j < chunk; ++j) {
-            const uint32_t r = r0 + j;
-            if (r >= nb) break;
-            const uint32_t c = h[nb - 1 - r];
-            if (need <= run + c) { s.res[0] = nb - 1 - r; s.res[1] = run; s.res[2] = c; break; }
-            run += c;
+    uint32_t seg = TK_WARPS, excl = 0;
+    {
+        uint32_t run = 0;
+#pragma unroll
+        for (int w = 0; w < TK_WARPS; ++w) {
+            const uint32_t v = s.scan[w];
+            if (seg == TK_WARPS && need <= run + v) { seg = w; excl = run; }
+            run += v;
         }
     }
     __syncthreads();
-}
-
-__device__ inline void load_hist(uint32_t* dst, const uint32_t* src, uint32_t nb) {
-    for (uint32_t i = threadIdx.x; i < nb; i += TK_THREADS) dst[i] = __ldcg(src + i);
+    if (seg == TK_WARPS) return;                       // fewer than `need` elements (uniform across the block)
+    // level 2: inside segment `seg`, warp w owns reversed positions [w*sublen, (w+1)*sublen), sublen <= 32
+    const uint32_t s0 = seg * seglen, s1 = min(nb, s0 + seglen);
+    const uint32_t sublen = (seglen + TK_WARPS - 1) / TK_WARPS;
+    const uint32_t r = s0 + warp * sublen + lane;
+    const bool live = lane < sublen && r < s1;
+    const uint32_t v = live ? __ldcg(h + (nb - 1 - r)) : 0u;
+    const uint32_t incl = warp_incl_scan(v);
+    if (lane == 31) s.scan[warp] = incl;
+    __syncthreads();
+    uint32_t sub = TK_WARPS, excl2 = excl;
+    {
+        uint32_t run = excl;
+#pragma unroll
+        for (int w = 0; w < TK_WARPS; ++w) {
+            const uint32_t t = s.scan[w];
+            if (sub == TK_WARPS && need <= run + t) { sub = w; excl2 = run; }
+            run += t;
+        }
+    }
+    if (warp == sub && live) {
+        const uint32_t before = excl2 + incl - v;
+        if (before < need && need <= before + v) { s.res[0] = nb - 1 - r; s.res[1] = before; s.res[2] = v; }
+    }
     __syncthreads();
 }
 
@@ -148,9 +165,13 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
     uint32_t* status = P.ctrl + CT_STATUS;
     const uint32_t nchunks = (d + TK_CHUNK - 1) / TK_CHUNK;
 
+    // phase time stamps of block 0 (low word of the nanosecond global timer), for profiling only
+#define SC_STAMP(i) do { if (gtid == 0) { uint32_t ts_; asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(ts_)); \
+                                          P.ctrl[CT_STAMP + (i)] = ts_; } } while (0)
 #define SC_BARRIER() do { if (!grid_barrier(P.barrier, nblocks, status, P.spin_limit, &s.flag)) return; } while (0)
 
     // ---------------- P0: clear scratch, sample ----------------------------------------------
+    SC_STAMP(0);
     zero_words(P.bitmap, size_t(P.ntiles) * 32, gtid, gsize);
     zero_words(P.fine_hist, NFINE, gtid, gsize);
     zero_words(P.digit_hist, DH_PASSES * DH_BINS, gtid, gsize);
@@ -179,16 +200,20 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
             if (h) atomicAdd(&P.samp_hist[i], h);
         }
     }
+    SC_STAMP(1);
     SC_BARRIER();
+    SC_STAMP(2);
 
     // ---------------- P1 + P2: bound from the sample, filter pass ----------------------------------
     bool fast = !P.force_exact;
     if (fast) {
-        load_hist(s.hist, P.samp_hist, NCOARSE);
-        find_from_top(s.hist, NCOARSE, P.samp_target, s);
+        find_from_top(P.samp_hist, NCOARSE, P.samp_target, s);
         b_lo = (s.res[0] == 0xFFFFFFFFu) ? 0u : s.res[0];
         __syncthreads();
+        SC_STAMP(3);
 
+        for (uint32_t i = tid; i <= WIN; i += TK_THREADS) s.cw[i] = 0;
+        __syncthreads();
         const uint32_t thr_key = b_lo << COARSE_SHIFT;
         const uint32_t fine_base = b_lo << (COARSE_SHIFT - FINE_SHIFT);
         uint2* stage = s.stage[warp];
@@ -229,7 +254,7 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
                         if (pred[c]) {
                             stage[wcnt + __popc(bal & ((1u << lane) - 1u))] = make_uint2(key[c], p + c);
                             const uint32_t cb = (key[c] >> COARSE_SHIFT) - b_lo;
-                            atomicAdd(&P.coarse_win[cb < WIN ? cb : WIN], 1u);
+                            atomicAdd(&s.cw[cb < WIN ? cb : WIN], 1u);
                             if (cb < WIN) atomicAdd(&P.fine_hist[(key[c] >> FINE_SHIFT) - fine_base], 1u);
                         }
                         wcnt += __popc(bal);
@@ -245,8 +270,15 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
             for (uint32_t i = lane; i < wcnt; i += 32)
                 if (gb + i < P.cand_cap) P.cand[gb + i] = stage[i];
         }
+        __syncthreads();
+        for (uint32_t i = tid; i <= WIN; i += TK_THREADS) {
+            const uint32_t h = s.cw[i];
+            if (h) atomicAdd(&P.coarse_win[i], h);
+        }
     }
+    SC_STAMP(4);
     SC_BARRIER();
+    SC_STAMP(5);
 
     // the sample histogram must be all zero again when the kernel ends
     if (!P.force_exact) zero_words(P.samp_hist, NCOARSE, gtid, gsize);
@@ -261,8 +293,7 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
         fast = (M >= k) && (M <= P.cand_cap);
     }
     if (fast) {
-        load_hist(s.hist, P.coarse_win, WIN + 1);
-        find_from_top(s.hist, WIN + 1, k, s);
+        find_from_top(P.coarse_win, WIN + 1, k, s);
         const uint32_t cb = s.res[0], above = s.res[1], at = s.res[2];
         __syncthreads();
         if (cb >= WIN) {
@@ -270,8 +301,7 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
         } else {
             st.prefix = b_lo + cb; st.nbits = 13; st.need = k - above; st.group = at;
             if (!sel_done(st)) {
-                load_hist(s.hist, P.fine_hist + cb * 512u, 512);
-                find_from_top(s.hist, 512, st.need, s);
+                find_from_top(P.fine_hist + cb * 512u, 512, st.need, s);
                 const uint32_t fb = s.res[0], fa = s.res[1], fc = s.res[2];
                 __syncthreads();
                 if (fb == 0xFFFFFFFFu) {
@@ -334,8 +364,7 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
             }
         }
         SC_BARRIER();
-        load_hist(s.hist, gh, 1u << W);
-        find_from_top(s.hist, 1u << W, st.need, s);
+        find_from_top(gh, 1u << W, st.need, s);
         const uint32_t dg = s.res[0], above = s.res[1], at = s.res[2];
         __syncthreads();
         if (dg == 0xFFFFFFFFu) {                                       // cannot happen: the group holds >= need
@@ -349,15 +378,24 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
     }
 
     // ---------------- P4: mark winners (composite >= T) ---------------------------------------------
+    SC_STAMP(6);
     const uint64_t T = st.nbits >= 62 ? st.prefix : (st.prefix << (62 - st.nbits));
     const uint32_t span_coords = P.tiles_per_block * TILE;
     if (fast) {
+        // winners per scan span are counted in shared memory first (nblocks <= NCOARSE spans)
+        for (uint32_t i = tid; i < nblocks; i += TK_THREADS) s.hist[i] = 0;
+        __syncthreads();
         for (size_t i = gtid; i < M; i += gsize) {
             const uint2 e = __ldcg(&P.cand[i]);
             if (composite(e.x, e.y) >= T) {
                 atomicOr(&P.bitmap[e.y >> 5], 1u << (e.y & 31u));
-                atomicAdd(&P.block_tot[e.y / span_coords], 1u);
+                atomicAdd(&s.hist[e.y / span_coords], 1u);
             }
+        }
+        __syncthreads();
+        for (uint32_t i = tid; i < nblocks; i += TK_THREADS) {
+            const uint32_t h = s.hist[i];
+            if (h) atomicAdd(&P.block_tot[i], h);
         }
     } else {
         // every 128-coordinate group is owned by one warp: whole bitmap words, plain stores
@@ -391,7 +429,9 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
             }
         }
     }
+    SC_STAMP(7);
     SC_BARRIER();
+    SC_STAMP(8);
 
     // ---------------- P5: scan the bitmap: tile prefixes and ascending indices ---------------------
     {
@@ -441,7 +481,9 @@ __global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkPa
             if (running != k) atomicCAS(status, DEV_OK, DEV_INTERNAL);  // the winners must number exactly k
         }
     }
+    SC_STAMP(9);
 #undef SC_BARRIER
+#undef SC_STAMP
 }
 
 }  // namespace sc
