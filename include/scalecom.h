@@ -168,6 +168,35 @@ int scalecom_query(scalecom_ctx* ctx, int item, int64_t* out);
  */
 int scalecom_kernel_ms(scalecom_ctx* ctx, float ms[3], int32_t* nsteps);
 
+/*
+ * Leader selection (step 2 only) for callers that cannot allocate device memory.
+ * The paper has no counterpart: this entry point exists for deployment reasons.
+ * A process whose GPU memory is already fully owned by a framework's caching
+ * allocator, or capped by a fixed partition, gets an error from cudaMalloc; a
+ * latency-critical loop cannot afford the device-wide synchronisation cudaMalloc
+ * implies.  Here the selection kernel's scratch is a fixed array inside the
+ * library image (about 8.4 MB, present on every GPU that loads the library for
+ * the life of the process), and the call performs no cudaMalloc, cudaFree or
+ * any other allocating call.
+ *   g, m        DEVICE fp32[d]: the leader's gradient and memory; keys are |m + g|.
+ *   d           1 <= d <= SCALECOM_STATIC_MAX_D (larger vectors: INVALID_ARG; use a handle).
+ *   k           1 <= k <= d.
+ *   out_idx     DEVICE int32[k], written: the same ascending index list scalecom_step returns.
+ *   dev_status  DEVICE int32, optional (NULL to skip): receives 0, or 5 if a bounded
+ *               in-kernel wait expired, or 7 if a consistency check failed (out_idx is
+ *               then undefined).
+ *   cuda_stream cudaStream_t as void*; the work is asynchronous on it, on the current device.
+ * The first call on each device looks up the array's device address and the
+ * kernel's launch limits; make that first call before any stream capture begins.
+ * All calls on a device share the one array, which still holds the previous
+ * call's contents: each call clears what must start at zero, and two calls whose
+ * GPU work overlaps (different streams, no dependency) race on it -- order them.
+ * Errors: NULL_PTR, INVALID_ARG, ALIAS, CUDA.
+ */
+#define SCALECOM_STATIC_MAX_D (1 << 20)
+int scalecom_topk_static(const float* g, const float* m, int64_t d, int64_t k, int32_t* out_idx,
+                         int32_t* dev_status, void* cuda_stream);
+
 /* Static, never NULL. */
 const char* scalecom_strerror(int code);
 

@@ -29,7 +29,9 @@ EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
     "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
+    "scalecom_topk_static",
 )
+STATIC_MAX_D = 1 << 20
 
 _lib = None
 
@@ -74,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.scalecom_query.argtypes = [vp, ctypes.c_int, ctypes.POINTER(i64)]
         L.scalecom_kernel_ms.restype = ctypes.c_int
         L.scalecom_kernel_ms.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(i32)]
+        L.scalecom_topk_static.restype = ctypes.c_int
+        L.scalecom_topk_static.argtypes = [vp, vp, i64, i64, vp, vp, vp]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -116,6 +120,12 @@ def scalecom_step_host(handle: int, host_grads: Sequence[int], mem: Sequence[int
 
 def scalecom_destroy(handle: Optional[int]) -> None:
     lib().scalecom_destroy(handle)
+
+
+def scalecom_topk_static(g: int, m: int, d: int, k: int, out_idx: int, dev_status: Optional[int],
+                         stream: Optional[int]) -> int:
+    """Raw mirror of the allocation-free selection entry point (device addresses as integers)."""
+    return lib().scalecom_topk_static(g, m, int(d), int(k), out_idx, dev_status, stream)
 
 
 # ---- tensor-level convenience wrapper ------------------------------------------------------------

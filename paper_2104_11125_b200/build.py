@@ -12,7 +12,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libscalecom.so")
 STAMP = LIB + ".srchash"
 
-SOURCES = ["scalecom.cu"]
+SOURCES = ["scalecom.cu", "topk_static.cu"]
 HEADERS = ["common.cuh", "topk_select.cuh", "learner_pass.cuh"]
 
 NVCC_FLAGS = [
