@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50")
+    ap.add_argument("--batches", type=int, default=MAX_BATCHES,
+                    help="distinct gradient batches kept in HBM (steps cycle through them); small values keep "
+                         "the footprint low for profiler captures")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -114,6 +117,22 @@ class ClockSampler(threading.Thread):
         s = sorted(self.samples)
         return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def job_value(n, d, world, ms_step):
+    """Whole-job learner-elements/s: every rank processed n*d learner-coordinates per step."""
+    return n * d * world / (ms_step * 1e-3)
+
+
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
 
 
 def cpu_threads():
@@ -204,7 +223,7 @@ def main():
     w = get_workload(args.workload)
     K, Wm = args.steps, max(args.warmup, 3)
     prof = W.profile(w, dev)
-    nb = min(K + Wm, MAX_BATCHES)
+    nb = max(1, min(K + Wm, args.batches, MAX_BATCHES))
     batches = [W.gradients(w, s, dev, prof) for s in range(nb)]
     mem = W.initial_memory(w, dev)
     theta = W.initial_weights(w, dev)
@@ -264,15 +283,11 @@ def main():
         e2e_ms = None
 
     # ---- max over ranks --------------------------------------------------------------------------------
-    if world > 1:
-        tt = torch.tensor([ms_total, e2e_ms or 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total, e2e_max = float(tt[0]), float(tt[1])
-        e2e_ms = e2e_max if e2e_ms is not None else None
+    ms_total, e2e_max = max_over_ranks([ms_total, e2e_ms or 0.0], dev)
+    e2e_ms = e2e_max if e2e_ms is not None else None
 
     if rank == 0:
         ms_step = ms_total / K
-        units = w.n * w.d * world
         peak, peak_src = measured_peak()
         lp_ms = kms[1] / max(ksteps, 1)
         tk_ms = kms[0] / max(ksteps, 1)
@@ -281,7 +296,7 @@ def main():
         lp_gbs = lp_bytes / (lp_ms * 1e-3) / 1e9
         tk_gbs = tk_bytes / (tk_ms * 1e-3) / 1e9
         out = {
-            "metric": METRIC, "value": units / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": job_value(w.n, w.d, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "n": w.n, "d": w.d, "k": w.k, "beta": w.beta, "lr": w.lr,
@@ -301,7 +316,7 @@ def main():
             "clocks": clocks,
         }
         if e2e_ms is not None:
-            out["e2e"] = {"value": units / (e2e_ms * 1e-3), "unit": UNIT,
+            out["e2e"] = {"value": job_value(w.n, w.d, world, e2e_ms), "unit": UNIT,
                           "h2d_bytes_per_step": 4 * w.n * w.d, "d2h_bytes_per_step": 8 * w.k,
                           "ms_per_step": e2e_ms, "api": "scalecom_step_host (pinned host gradients in, idx/val out)"}
         if world == 1 and not args.no_cpu_baseline:

@@ -95,7 +95,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned long long* counter, uint32
         __threadfence();
         const unsigned long long old = atomicAdd(counter, 1ULL);
         const unsigned long long target = (old / nblocks + 1ULL) * nblocks;
-        for (uint32_t it = 0; it <= spin_limit; ++it) {
+        for (uint32_t it = 0; it < spin_limit; ++it) {   // a limit of 0 expires at once
             if (ld_acquire_u64(counter) >= target) { ok = 1; break; }
             if (ld_relaxed_u32(status) != DEV_OK) break;
             if (it > 64) __nanosleep(it > 4096 ? 256 : 32);

@@ -158,6 +158,7 @@ def _draw(w: Workload, prof: Profile, gen: torch.Generator, device) -> torch.Ten
     if prof.laplace is not None:
         x.mul_(prof.sigma)
         u = torch.rand(w.d, generator=gen, device=device, dtype=torch.float32).sub_(0.5)
+        u.clamp_(-0.49999997, 0.49999997)                  # keeps log1p finite: |x| <= 16.7 b
         lap = torch.sign(u).mul_(torch.log1p(-2.0 * u.abs()).mul_(-prof.b))
         x = torch.where(prof.laplace, lap, x)
     elif prof.scale is not None:

@@ -151,3 +151,50 @@ def test_host_buffer_entry_point():
         assert ctx.status() == 0
     assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(m, m_o))
     assert np.array_equal(th.cpu().numpy(), th_o)
+
+
+def test_bounded_wait_expiry_is_reported_and_recoverable():
+    """Failure detection without a GPU fault: with the barrier's iteration bound set to 0 every
+    wait gives up at once, the kernel returns, the status word says TIMEOUT, the handle refuses
+    work until it is reset, and after the reset results are right again."""
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    w = W.TINY.scaled(200_000)                      # 25 blocks in the selection kernel
+    prof = W.profile(w, DEV)
+    g = W.gradients(w, 0, DEV, prof)
+    idx = torch.empty(w.k, device=DEV, dtype=torch.int32)
+    val = torch.empty(w.k, device=DEV)
+    with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
+        assert ctx.query(binding.Q_TOPK_BLOCKS) > 1
+        ctx.set_option(binding.OPT_SPIN_LIMIT, 0)
+        m = W.initial_memory(w, DEV)
+        ctx.step(g, m, None, 0, idx, val)
+        assert ctx.status() == binding.ERR_TIMEOUT
+        with pytest.raises(sc.ScaleComError) as ei:
+            ctx.step(g, m, None, 0, idx, val)
+        assert ei.value.code == binding.ERR_BAD_STATE
+        ctx.set_option(binding.OPT_SPIN_LIMIT, 1 << 22)
+        ctx.reset()
+        assert ctx.status() == 0
+    _parity().workload_case(w, 2, DEV)              # a fresh handle on the same device is unaffected
+
+
+def test_argument_checks_on_device_pointers():
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding as b
+    d, n, k = 1000, 2, 10
+    g = [torch.zeros(d, device=DEV) for _ in range(n)]
+    m = [torch.zeros(d, device=DEV) for _ in range(n)]
+    idx = torch.empty(k, device=DEV, dtype=torch.int32)
+    val = torch.empty(k, device=DEV)
+    with sc.Context(d, n, k, 0.5, 0.1) as ctx:
+        h = ctx._h
+        gp, mp = [x.data_ptr() for x in g], [x.data_ptr() for x in m]
+        assert b.scalecom_step(h, gp, mp, None, -1, idx.data_ptr(), val.data_ptr()) == b.ERR_INVALID_ARG
+        assert b.scalecom_step(h, gp, [mp[0], gp[1]], None, 0, idx.data_ptr(), val.data_ptr()) == b.ERR_ALIAS
+        assert b.scalecom_step(h, gp, [mp[0], mp[0]], None, 0, idx.data_ptr(), val.data_ptr()) == b.ERR_ALIAS
+        assert b.scalecom_step(h, gp, mp, mp[0], 0, idx.data_ptr(), val.data_ptr()) == b.ERR_ALIAS
+        assert b.scalecom_step(h, gp, mp, None, 0, None, val.data_ptr()) == b.ERR_NULL_PTR
+        assert b.scalecom_step(h, [gp[0], None], mp, None, 0, idx.data_ptr(), val.data_ptr()) == b.ERR_NULL_PTR
+        assert ctx.query(b.Q_KERNEL_LAUNCHES) == 0          # nothing was launched by the rejected calls
+        assert ctx.status() == 0
