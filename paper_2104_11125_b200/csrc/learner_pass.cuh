@@ -14,8 +14,15 @@
 
 namespace sc {
 
+#ifndef SC_LP_UNROLL
+#define SC_LP_UNROLL 8
+#endif
+#ifndef SC_LP_BLOCKS_PER_SM
+#define SC_LP_BLOCKS_PER_SM 2
+#endif
 constexpr int LP_THREADS = 256;            // x 4 coordinates = one tile
-constexpr int LP_UNROLL = 4;               // learners in flight per thread
+constexpr int LP_UNROLL = SC_LP_UNROLL;    // learners in flight per thread
+constexpr int LP_BLOCKS_PER_SM = SC_LP_BLOCKS_PER_SM;
 
 template <int N>
 struct PtrTable {
@@ -32,16 +39,24 @@ struct LearnerParams {
     float* out_val;                        // [k]
     float* gathered;                       // [n * k] or nullptr
     float* weights;                        // [d] or nullptr (then Algorithm 1 line 12 is not applied here)
+    unsigned long long* span;              // nullptr, or {min start, max end} of all blocks on the ns global timer (profiling)
 };
 
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
 template <int N, bool VEC>
-__global__ void __launch_bounds__(LP_THREADS, 4)
+__global__ void __launch_bounds__(LP_THREADS, LP_BLOCKS_PER_SM)
 learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P) {
     const uint32_t tid = threadIdx.x, lane = lane_id();
     const uint32_t d = P.d;
     const int n = P.n;
     const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside the tile
     const uint32_t sh = (tid & 7u) * 4u;           // and its first bit inside that word
+    if (P.span && tid == 0) atomicMin(&P.span[0], global_timer_ns());
 
     for (uint32_t tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         // selection bits of this thread's four coordinates and the rank of the first selected one
@@ -96,6 +111,10 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                     if (P.weights) P.weights[p + c] = __fsub_rn(P.weights[p + c], __fmul_rn(P.lr, v));   // line 12
                 }
         }
+    }
+    if (P.span) {
+        __syncthreads();
+        if (tid == 0) atomicMax(&P.span[1], global_timer_ns());
     }
 }
 

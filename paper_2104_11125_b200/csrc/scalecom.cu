@@ -42,6 +42,7 @@ struct scalecom_ctx {
     bool timing = false;
     bool fuse_update = true;
     float* gathered = nullptr;
+    unsigned long long* lp_span = nullptr;   // experiment
 
     // host-buffer entry point
     float* stage_g = nullptr;          // n*d
@@ -170,6 +171,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     lp.out_val = out_val;
     lp.gathered = c->gathered;
     lp.weights = (weights && c->fuse_update) ? weights : nullptr;
+    lp.span = c->lp_span;
 
     bool vec_all = true;
     for (int i = 0; i < c->n; ++i) vec_all = vec_all && aligned16(grads[i]) && aligned16(mem[i]);
@@ -236,7 +238,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
         delete c;
         return SCALECOM_ERR_CUDA;
     }
-    if (occ_topk > 2) occ_topk = 2;
+    if (occ_topk > TK_BLOCKS_PER_SM) occ_topk = TK_BLOCKS_PER_SM;
 
     c->ntiles = uint32_t((d + TILE - 1) / TILE);
     // persistent selection grid: every resident slot, but no more blocks than there are chunks of work
@@ -385,6 +387,7 @@ int scalecom_set_stream(scalecom_ctx* c, void* cuda_stream) {
     return SCALECOM_OK;
 }
 
+int scalecom_experiment_span(scalecom_ctx* c, unsigned long long* p) { c->lp_span = p; return 0; }
 int scalecom_set_gathered(scalecom_ctx* c, float* dev_gathered) {
     if (!c) return SCALECOM_ERR_NULL_PTR;
     c->gathered = dev_gathered;

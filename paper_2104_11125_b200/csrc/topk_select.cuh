@@ -26,7 +26,14 @@
 
 namespace sc {
 
-constexpr int TK_THREADS = 512;
+#ifndef SC_TK_THREADS
+#define SC_TK_THREADS 512
+#endif
+#ifndef SC_TK_BLOCKS_PER_SM
+#define SC_TK_BLOCKS_PER_SM 2
+#endif
+constexpr int TK_THREADS = SC_TK_THREADS;
+constexpr int TK_BLOCKS_PER_SM = SC_TK_BLOCKS_PER_SM;
 constexpr int TK_WARPS = TK_THREADS / 32;
 constexpr int TK_UNROLL = 4;                                   // quads of g and of m in flight per thread
 constexpr uint32_t TK_CHUNK = TK_THREADS * 4 * TK_UNROLL;      // coordinates per block iteration (8192)
@@ -153,7 +160,7 @@ struct SelState {
 __device__ __forceinline__ bool sel_done(const SelState& st) { return st.group == st.need || st.nbits >= 62; }
 
 template <bool VEC>
-__global__ void __launch_bounds__(TK_THREADS, 2) topk_select_kernel(const TopkParams P) {
+__global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kernel(const TopkParams P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TopkShared& s = *reinterpret_cast<TopkShared*>(smem_raw);
 

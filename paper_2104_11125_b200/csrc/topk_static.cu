@@ -69,7 +69,7 @@ int setup_device(int dev, DeviceSetup& su) {
         return SCALECOM_ERR_CUDA;
     if (o2 < occ) occ = o2;
     if (occ < 1) return SCALECOM_ERR_CUDA;
-    if (occ > 2) occ = 2;
+    if (occ > TK_BLOCKS_PER_SM) occ = TK_BLOCKS_PER_SM;
     su.scratch = static_cast<unsigned char*>(p);
     su.max_blocks = sms * occ;
     if (su.max_blocks > int(MAX_BLOCKS)) su.max_blocks = int(MAX_BLOCKS);
