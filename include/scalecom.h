@@ -145,11 +145,15 @@ int scalecom_reset(scalecom_ctx* ctx);
 #define SCALECOM_OPT_SPIN_LIMIT       2  /* iteration bound of the in-kernel grid barrier wait (>= 0)       */
 #define SCALECOM_OPT_KERNEL_TIMING    3  /* 1: bracket each kernel of a step with CUDA events                */
 #define SCALECOM_OPT_FUSE_UPDATE      4  /* 1 (default): step 5 runs inside the learner pass; 0: own kernel  */
+#define SCALECOM_OPT_USE_HINT         5  /* 1 (default): a step starts its pre-filter from the threshold the
+                                            previous step of this handle found; 0: always sample afresh.
+                                            Affects speed only, never results                              */
 int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 
 /* Items for scalecom_query (each synchronises the stream when it reads device state). */
 #define SCALECOM_Q_WORKSPACE_BYTES  1  /* device bytes owned by the handle                                    */
-#define SCALECOM_Q_LAST_TOPK_PATH   2  /* last step's selection path: 0 = sampled pre-filter, 1 = full select */
+#define SCALECOM_Q_LAST_TOPK_PATH   2  /* last step's selection path: 0 = sampled pre-filter, 1 = full select,
+                                          2 = pre-filter started from the previous step's threshold           */
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */
@@ -175,7 +179,7 @@ int scalecom_kernel_ms(scalecom_ctx* ctx, float ms[3], int32_t* nsteps);
  * allocator, or capped by a fixed partition, gets an error from cudaMalloc; a
  * latency-critical loop cannot afford the device-wide synchronisation cudaMalloc
  * implies.  Here the selection kernel's scratch is a fixed array inside the
- * library image (about 8.4 MB, present on every GPU that loads the library for
+ * library image (about 11 MB, present on every GPU that loads the library for
  * the life of the process), and the call performs no cudaMalloc, cudaFree or
  * any other allocating call.
  *   g, m        DEVICE fp32[d]: the leader's gradient and memory; keys are |m + g|.

@@ -63,19 +63,31 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
     return v;
 }
 
-__device__ __forceinline__ uint32_t warp_sum(uint32_t v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
-    return v;
-}
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v) { return __reduce_add_sync(FULL, v); }
 
-// ---- bounded grid barrier ----------------------------------------------------------------------
+// ---- optional in-kernel time spans (build with -DSC_PROFILE_SPANS) -----------------------------------
+// Each kernel then takes a device pointer to {earliest block start, latest block end} on the
+// nanosecond global timer, which separates kernel time from launch gaps and event overhead.
+#ifdef SC_PROFILE_SPANS
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define SC_SPAN_BEGIN(sp) do { if ((sp) && threadIdx.x == 0) atomicMin(&(sp)[0], global_timer_ns()); } while (0)
+#define SC_SPAN_END(sp) do { if (sp) { __syncthreads(); if (threadIdx.x == 0) atomicMax(&(sp)[1], global_timer_ns()); } } while (0)
+#else
+#define SC_SPAN_BEGIN(sp) do { } while (0)
+#define SC_SPAN_END(sp) do { } while (0)
+#endif
+
+// ---- bounded grid barrier -----------------------------------------------------------------------
 // All blocks of a cooperative launch call this the same number of times.  The
-// 64-bit counter only ever grows; each arrival derives its own release value, so
-// no reset between barriers or launches is needed as long as every launch
-// completes (the host zeroes the counter after a device error).  The wait is
-// bounded: on expiry the status word becomes DEV_TIMEOUT, every waiter sees it
-// and the function returns false; callers then return without touching memory.
+// 64-bit arrival counter only ever grows; each arrival derives its own release
+// value from it, so nothing needs resetting between barriers or launches as long
+// as every launch completes (the host zeroes the counter after a device error).
+// The wait is bounded: on expiry the status word becomes DEV_TIMEOUT, every
+// waiter sees it and the function returns false; callers then return at once.
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
     unsigned long long v;
     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -87,20 +99,26 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p) {
     return v;
 }
 
-__device__ __forceinline__ bool grid_barrier(unsigned long long* counter, uint32_t nblocks,
-                                             uint32_t* status, uint32_t spin_limit, int* smem_flag) {
+struct GridBarrier {
+    unsigned long long* arrive;
+    uint32_t nblocks;
+    uint32_t* status;
+    uint32_t spin_limit;       // 0: every wait expires at once
+};
+
+__device__ __forceinline__ bool grid_barrier(const GridBarrier& gb, int* smem_flag) {
     __syncthreads();
     if (threadIdx.x == 0) {
         int ok = 0;
         __threadfence();
-        const unsigned long long old = atomicAdd(counter, 1ULL);
-        const unsigned long long target = (old / nblocks + 1ULL) * nblocks;
-        for (uint32_t it = 0; it < spin_limit; ++it) {   // a limit of 0 expires at once
-            if (ld_acquire_u64(counter) >= target) { ok = 1; break; }
-            if (ld_relaxed_u32(status) != DEV_OK) break;
+        const unsigned long long old = atomicAdd(gb.arrive, 1ULL);
+        const unsigned long long target = (old / gb.nblocks + 1ULL) * gb.nblocks;
+        for (uint32_t it = 0; it < gb.spin_limit; ++it) {
+            if (ld_acquire_u64(gb.arrive) >= target) { ok = 1; break; }
+            if (ld_relaxed_u32(gb.status) != DEV_OK) break;
             if (it > 64) __nanosleep(it > 4096 ? 256 : 32);
         }
-        if (!ok) atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+        if (!ok) atomicCAS(gb.status, DEV_OK, DEV_TIMEOUT);
         __threadfence();
         *smem_flag = ok;
     }

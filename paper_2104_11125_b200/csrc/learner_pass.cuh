@@ -37,16 +37,13 @@ struct LearnerParams {
     const uint32_t* bitmap;                // [ntiles * 32]
     const uint32_t* tile_prefix;           // [ntiles + 1]
     float* out_val;                        // [k]
+    int32_t* out_idx;                      // [k]: the ascending index list, written here from the ranks
     float* gathered;                       // [n * k] or nullptr
     float* weights;                        // [d] or nullptr (then Algorithm 1 line 12 is not applied here)
-    unsigned long long* span;              // nullptr, or {min start, max end} of all blocks on the ns global timer (profiling)
+#ifdef SC_PROFILE_SPANS
+    unsigned long long* spans;             // {earliest block start, latest block end}, ns
+#endif
 };
-
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 
 template <int N, bool VEC>
 __global__ void __launch_bounds__(LP_THREADS, LP_BLOCKS_PER_SM)
@@ -56,7 +53,9 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
     const int n = P.n;
     const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside the tile
     const uint32_t sh = (tid & 7u) * 4u;           // and its first bit inside that word
-    if (P.span && tid == 0) atomicMin(&P.span[0], global_timer_ns());
+#ifdef SC_PROFILE_SPANS
+    SC_SPAN_BEGIN(P.spans);
+#endif
 
     for (uint32_t tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
         // selection bits of this thread's four coordinates and the rank of the first selected one
@@ -107,15 +106,15 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
             for (int c = 0; c < 4; ++c)
                 if ((nib >> c) & 1u) {
                     const float v = __fdiv_rn(sum[c], P.nf);                           // line 10: one division by n
+                    P.out_idx[r] = int32_t(p + c);
                     P.out_val[r++] = v;
                     if (P.weights) P.weights[p + c] = __fsub_rn(P.weights[p + c], __fmul_rn(P.lr, v));   // line 12
                 }
         }
     }
-    if (P.span) {
-        __syncthreads();
-        if (tid == 0) atomicMax(&P.span[1], global_timer_ns());
-    }
+#ifdef SC_PROFILE_SPANS
+    SC_SPAN_END(P.spans);
+#endif
 }
 
 // Algorithm 1 line 12 as its own kernel: theta[idx[j]] -= lr * val[j].

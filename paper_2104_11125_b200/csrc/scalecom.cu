@@ -28,7 +28,8 @@ struct scalecom_ctx {
     uint32_t *block_tot = nullptr, *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr;
     unsigned long long* barrier = nullptr;
     uint2* cand = nullptr;
-    uint32_t cand_cap = 0, ntiles = 0, tiles_per_block = 0;
+    uint2* blist = nullptr;
+    uint32_t seg_cap = 0, ntiles = 0, tiles_per_block = 0;
     size_t ctrl_region_bytes = 0;      // prefix of the workspace that reset() clears
 
     // launch geometry
@@ -38,11 +39,12 @@ struct scalecom_ctx {
 
     // options
     uint32_t force_exact = 0;
+    uint32_t use_hint = 1;
     uint32_t spin_limit = 1u << 22;
     bool timing = false;
     bool fuse_update = true;
     float* gathered = nullptr;
-    unsigned long long* lp_span = nullptr;   // experiment
+    unsigned long long* spans = nullptr;     // only used by SC_PROFILE_SPANS builds
 
     // host-buffer entry point
     float* stage_g = nullptr;          // n*d
@@ -53,6 +55,7 @@ struct scalecom_ctx {
     static constexpr int EV_RING = 256;
     cudaEvent_t* ev = nullptr;         // [EV_RING * 4], created when timing is first switched on
     int64_t ev_steps = 0;              // steps recorded since the last read
+    bool ev_has_update[EV_RING] = {};  // whether the step recorded the fourth event
     bool poisoned = false;
     int64_t launches = 0;
 };
@@ -141,6 +144,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     tp.samp_stride = c->samp_stride;
     tp.samp_target = c->samp_target;
     tp.force_exact = c->force_exact;
+    tp.use_hint = c->use_hint;
     tp.spin_limit = c->spin_limit;
     tp.samp_hist = c->samp_hist;
     tp.coarse_win = c->coarse_win;
@@ -150,12 +154,16 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     tp.ctrl = c->ctrl;
     tp.barrier = c->barrier;
     tp.cand = c->cand;
-    tp.cand_cap = c->cand_cap;
+    tp.seg_cap = c->seg_cap;
+    tp.blist = c->blist;
     tp.bitmap = c->bitmap;
     tp.tile_prefix = c->tile_prefix;
     tp.ntiles = c->ntiles;
     tp.tiles_per_block = c->tiles_per_block;
-    tp.out_idx = out_idx;
+    tp.out_idx = nullptr;          // the learner pass writes the index list from the ranks it computes anyway
+#ifdef SC_PROFILE_SPANS
+    tp.spans = c->spans;
+#endif
 
     LearnerParams lp;
     lp.d = uint32_t(c->d);
@@ -169,9 +177,12 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     lp.bitmap = c->bitmap;
     lp.tile_prefix = c->tile_prefix;
     lp.out_val = out_val;
+    lp.out_idx = out_idx;
     lp.gathered = c->gathered;
     lp.weights = (weights && c->fuse_update) ? weights : nullptr;
-    lp.span = c->lp_span;
+#ifdef SC_PROFILE_SPANS
+    lp.spans = c->spans ? c->spans + 2 : nullptr;
+#endif
 
     bool vec_all = true;
     for (int i = 0; i < c->n; ++i) vec_all = vec_all && aligned16(grads[i]) && aligned16(mem[i]);
@@ -196,7 +207,9 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
         ++c->launches;
     }
     if (tm) {
-        if (cudaEventRecord(ev[3], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+        // without a separate update kernel the third interval is empty: one event fewer on the stream
+        c->ev_has_update[c->ev_steps % scalecom_ctx::EV_RING] = weights && !c->fuse_update;
+        if (weights && !c->fuse_update && cudaEventRecord(ev[3], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
         ++c->ev_steps;
     }
     return SCALECOM_OK;
@@ -268,19 +281,23 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
         }
     }
     {
-        int64_t cap = 3 * k + 16384;
-        if (cap > d) cap = d;
-        c->cand_cap = uint32_t(cap);
+        // candidate segment per warp of the selection grid: room for 4k survivors overall plus slack
+        // for uneven spread, never more than the warp's share of the vector
+        const int64_t warps = int64_t(c->topk_blocks) * TK_WARPS;
+        int64_t cap = (4 * k + warps - 1) / warps + 32;
+        const int64_t share = (d + warps - 1) / warps + 32;
+        if (cap > share) cap = share;
+        c->seg_cap = uint32_t(cap);
     }
 
     // carve the workspace; the first region (histograms, counters) is what reset() clears
     size_t off = 0;
     auto carve = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
-    const size_t o_samp = carve(NCOARSE * 4), o_cw = carve((WIN + 1) * 4), o_ctrl = carve(CT_WORDS * 4), o_bar = carve(8);
+    const size_t o_samp = carve(NCOARSE * 4), o_cw = carve((WIN + 1) * 4), o_ctrl = carve(CT_WORDS * 4), o_bar = carve(256);
     const size_t o_bt = carve(size_t(c->topk_blocks) * 4);
-    c->ctrl_region_bytes = off;
     const size_t o_fine = carve(NFINE * 4), o_dh = carve(size_t(DH_PASSES) * DH_BINS * 4);
-    const size_t o_cand = carve(size_t(c->cand_cap) * 8);
+    c->ctrl_region_bytes = off;                 // everything the kernel expects to find zero
+    const size_t o_cand = carve(size_t(c->seg_cap) * c->topk_blocks * TK_WARPS * 8), o_bl = carve(size_t(BCAP) * 8);
     const size_t o_bm = carve(size_t(c->ntiles) * 32 * 4), o_tp = carve((size_t(c->ntiles) + 1) * 4);
     c->ws_bytes = off;
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
@@ -297,6 +314,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->fine_hist = reinterpret_cast<uint32_t*>(base + o_fine);
     c->digit_hist = reinterpret_cast<uint32_t*>(base + o_dh);
     c->cand = reinterpret_cast<uint2*>(base + o_cand);
+    c->blist = reinterpret_cast<uint2*>(base + o_bl);
     c->bitmap = reinterpret_cast<uint32_t*>(base + o_bm);
     c->tile_prefix = reinterpret_cast<uint32_t*>(base + o_tp);
 
@@ -387,7 +405,11 @@ int scalecom_set_stream(scalecom_ctx* c, void* cuda_stream) {
     return SCALECOM_OK;
 }
 
-int scalecom_experiment_span(scalecom_ctx* c, unsigned long long* p) { c->lp_span = p; return 0; }
+#ifdef SC_PROFILE_SPANS
+// Profiling builds only: p points to 4 device u64 {selection start, end, learner pass start, end}
+// (initialise starts to a large value, ends to 0); nullptr switches the time spans off.
+int scalecom_profile_spans(scalecom_ctx* c, unsigned long long* p) { c->spans = p; return 0; }
+#endif
 int scalecom_set_gathered(scalecom_ctx* c, float* dev_gathered) {
     if (!c) return SCALECOM_ERR_NULL_PTR;
     c->gathered = dev_gathered;
@@ -451,6 +473,7 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
             return SCALECOM_OK;
         }
         case SCALECOM_OPT_FUSE_UPDATE: c->fuse_update = value != 0; return SCALECOM_OK;
+        case SCALECOM_OPT_USE_HINT: c->use_hint = value ? 1u : 0u; return SCALECOM_OK;
         default: return SCALECOM_ERR_INVALID_ARG;
     }
 }
@@ -473,7 +496,7 @@ int scalecom_query(scalecom_ctx* c, int item, int64_t* out) {
             *out = item == SCALECOM_Q_LAST_TOPK_PATH ? w[CT_PATH] : w[CT_M];
             return SCALECOM_OK;
         default:
-            if (item >= SCALECOM_Q_PHASE_STAMP0 && item < SCALECOM_Q_PHASE_STAMP0 + CT_NSTAMPS) {
+            if (item >= SCALECOM_Q_PHASE_STAMP0 && item < SCALECOM_Q_PHASE_STAMP0 + 16) {
                 if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
                     cudaMemcpy(w, c->ctrl, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess)
                     return SCALECOM_ERR_CUDA;
@@ -493,7 +516,8 @@ int scalecom_kernel_ms(scalecom_ctx* c, float ms[3], int32_t* nsteps) {
     ms[0] = ms[1] = ms[2] = 0.f;
     for (int64_t s = c->ev_steps - kept; s < c->ev_steps; ++s) {
         cudaEvent_t* ev = c->ev + 4 * (s % scalecom_ctx::EV_RING);
-        for (int i = 0; i < 3; ++i) {
+        const int nint = c->ev_has_update[s % scalecom_ctx::EV_RING] ? 3 : 2;
+        for (int i = 0; i < nint; ++i) {
             float x = 0.f;
             if (cudaEventElapsedTime(&x, ev[i], ev[i + 1]) != cudaSuccess) return SCALECOM_ERR_CUDA;
             ms[i] += x;

@@ -21,7 +21,7 @@ namespace {
 
 constexpr uint32_t MAX_D = SCALECOM_STATIC_MAX_D;
 constexpr uint32_t MAX_TILES = (MAX_D + TILE - 1) / TILE;
-constexpr uint32_t MAX_BLOCKS = 4096;
+constexpr uint32_t MAX_BLOCKS = 512;
 constexpr int MAX_DEVICES = 64;
 
 constexpr size_t al(size_t x) { return (x + 255) / 256 * 256; }
@@ -30,16 +30,18 @@ constexpr size_t OFF_SAMP = 0;
 constexpr size_t OFF_CW = OFF_SAMP + al(NCOARSE * 4);
 constexpr size_t OFF_CTRL = OFF_CW + al((WIN + 1) * 4);
 constexpr size_t OFF_BAR = OFF_CTRL + al(CT_WORDS * 4);
-constexpr size_t OFF_BT = OFF_BAR + al(8);
-constexpr size_t OFF_CLEAR_END = OFF_BT + al(MAX_BLOCKS * 4);
-constexpr size_t OFF_FINE = OFF_CLEAR_END;
+constexpr size_t OFF_BT = OFF_BAR + al(256);
+constexpr size_t OFF_FINE = OFF_BT + al(MAX_BLOCKS * 4);
 constexpr size_t OFF_DH = OFF_FINE + al(NFINE * 4);
-constexpr size_t OFF_BM = OFF_DH + al(size_t(DH_PASSES) * DH_BINS * 4);
+constexpr size_t OFF_CLEAR_END = OFF_DH + al(size_t(DH_PASSES) * DH_BINS * 4);
+constexpr size_t OFF_BM = OFF_CLEAR_END;
 constexpr size_t OFF_TP = OFF_BM + al(size_t(MAX_TILES) * 32 * 4);
-constexpr size_t OFF_CAND = OFF_TP + al((size_t(MAX_TILES) + 1) * 4);
-constexpr size_t SCRATCH_BYTES = OFF_CAND + al(size_t(MAX_D) * 8);
+constexpr size_t OFF_BL = OFF_TP + al((size_t(MAX_TILES) + 1) * 4);
+constexpr size_t OFF_CAND = OFF_BL + al(size_t(BCAP) * 8);
+constexpr size_t CAND_ENTRIES = size_t(MAX_D) + 32u * MAX_BLOCKS * TK_WARPS;   // every warp's share of the vector + slack
+constexpr size_t SCRATCH_BYTES = OFF_CAND + al(CAND_ENTRIES * 8);
 
-// About 8.4 MB, held by every GPU that loads the library until the process exits.
+// About 11 MB, held by every GPU that loads the library until the process exits.
 // In host code this name is only a stand-in for the symbol, never a device
 // address: the address the kernel gets comes from cudaGetSymbolAddress below.
 static __device__ __align__(256) unsigned char g_scratch[SCRATCH_BYTES];
@@ -121,6 +123,7 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
         }
     }
     P.force_exact = 0;
+    P.use_hint = 0;               // the scratch is shared by unrelated callers: no carry-over between calls
     P.spin_limit = 1u << 22;
     P.samp_hist = reinterpret_cast<uint32_t*>(base + OFF_SAMP);
     P.coarse_win = reinterpret_cast<uint32_t*>(base + OFF_CW);
@@ -132,22 +135,30 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
     P.bitmap = reinterpret_cast<uint32_t*>(base + OFF_BM);
     P.tile_prefix = reinterpret_cast<uint32_t*>(base + OFF_TP);
     P.cand = reinterpret_cast<uint2*>(base + OFF_CAND);
-    {
-        int64_t cap = 3 * k + 16384;
-        if (cap > d) cap = d;
-        P.cand_cap = uint32_t(cap);
-    }
+    P.blist = reinterpret_cast<uint2*>(base + OFF_BL);
     P.ntiles = uint32_t((d + TILE - 1) / TILE);
     const uint32_t chunks = uint32_t((d + TK_CHUNK - 1) / TK_CHUNK);
     uint32_t blocks = uint32_t(su.max_blocks);
     if (blocks > chunks) blocks = chunks;
     if (blocks < 1) blocks = 1;
+    {
+        // one candidate segment per warp, carved from the fixed candidate area
+        const int64_t warps = int64_t(blocks) * TK_WARPS;
+        int64_t cap = (4 * k + warps - 1) / warps + 32;
+        const int64_t share = (d + warps - 1) / warps + 32;
+        if (cap > share) cap = share;
+        if (cap * warps > int64_t(CAND_ENTRIES)) cap = int64_t(CAND_ENTRIES) / warps;
+        P.seg_cap = uint32_t(cap);
+    }
     P.tiles_per_block = (P.ntiles + blocks - 1) / blocks;
     P.out_idx = out_idx;
+#ifdef SC_PROFILE_SPANS
+    P.spans = nullptr;
+#endif
 
     // Every call shares the array and finds the previous call's contents in it: the
-    // counters, the sample histogram and the barrier word must start at zero (the
-    // kernel itself clears the rest before using it).
+    // counters, the histograms and the barrier word must start at zero (the kernel
+    // itself clears the rest before using it).
     if (cudaMemsetAsync(base, 0, OFF_CLEAR_END, stream) != cudaSuccess) { cudaGetLastError(); return SCALECOM_ERR_CUDA; }
     const bool vec = ((reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(m)) & 15u) == 0;
     void* args[] = {&P};

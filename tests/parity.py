@@ -42,7 +42,7 @@ def assert_step_matches(tag, idx_g, val_g, G_g, m_g, th_g, idx_o, val_o, G_o, m_
 
 
 def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exact=False, fuse_update=True,
-                    want_path=None, offset=0, tag="case"):
+                    want_path=None, offset=0, use_hint=True, tag="case"):
     """grads_per_step: list over steps of lists of n CUDA fp32 tensors.
     m0: list of n CUDA tensors (initial memory), theta0: CUDA tensor or None.
     offset > 0 places every device vector `offset` floats past a 16-byte boundary
@@ -70,6 +70,7 @@ def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exac
         ctx.set_gathered(G)
         ctx.set_option(binding.OPT_FORCE_EXACT_PATH, int(force_exact))
         ctx.set_option(binding.OPT_FUSE_UPDATE, int(fuse_update))
+        ctx.set_option(binding.OPT_USE_HINT, int(use_hint))
         for s, grads in enumerate(grads_per_step):
             t = t0 + s
             g_dev = [place(g) for g in grads]
@@ -84,7 +85,10 @@ def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exac
                                 th_g.cpu().numpy() if th_g is not None else None,
                                 idx_o, val_o, G_o, m_o, th_o)
     if want_path is not None:
-        assert all(p == want_path for p in paths), "%s: selection paths %s, wanted %d" % (tag, paths, want_path)
+        # 0 asks for the pre-filter path, whether it started from a fresh sample (0) or from the
+        # previous step's threshold (2); 1 asks for the exact path
+        good = (binding.PATH_SAMPLED, binding.PATH_HINTED) if want_path == 0 else (want_path,)
+        assert all(p in good for p in paths), "%s: selection paths %s, wanted %s" % (tag, paths, good)
     return paths
 
 

@@ -47,7 +47,8 @@ def fullsize_case(w, steps=2):
             g = W.gradients(w, t, DEV, prof)
             ctx.step(g, m_g, th_g, t, idx, val)
             assert ctx.status() == 0
-            assert ctx.query(binding.Q_LAST_TOPK_PATH) == 0, "expected the sampled pre-filter path"
+            path = ctx.query(binding.Q_LAST_TOPK_PATH)
+            assert path == (binding.PATH_SAMPLED if t == 0 else binding.PATH_HINTED), "step %d took path %d" % (t, path)
             L = t % n
             # ---- selection: full, bit-exact ----
             acc = oracle.accumulate(g[L].cpu().numpy(), m_full[L])

@@ -97,6 +97,8 @@ def test_ties_straddling_rank_k_on_the_fast_path():
     x[ties] = np.where(rng.random(600) < 0.5, tau, -tau)        # ~600 copies of the k-th magnitude
     paths = _edge([x, 0.9 * x, 1.1 * x], k, steps=3, tag="ties-at-k")
     assert paths[0] == 0
+    paths = _edge([x, 0.9 * x, 1.1 * x], k, steps=3, use_hint=False, tag="ties-at-k-nohint")
+    assert paths == [0, 0, 0]
 
 
 def test_many_learners_small_vector():
@@ -198,3 +200,24 @@ def test_argument_checks_on_device_pointers():
         assert b.scalecom_step(h, [gp[0], None], mp, None, 0, idx.data_ptr(), val.data_ptr()) == b.ERR_NULL_PTR
         assert ctx.query(b.Q_KERNEL_LAUNCHES) == 0          # nothing was launched by the rejected calls
         assert ctx.status() == 0
+
+
+def test_threshold_hint_is_used_then_survives_scale_jumps():
+    """The pre-filter bound carried over from the previous step only changes speed.  Stationary
+    gradients take the hinted path from the second step on; a jump of the gradient scale makes the
+    hint useless (too few or far too many survivors) and the step falls back to a fresh sample."""
+    from paper_2104_11125_b200 import binding
+    w = W.TINY.scaled(600_011)
+    prof = W.profile(w, DEV)
+    base = [W.gradients(w, s, DEV, prof) for s in range(6)]
+    p = _parity()
+    # beta = 0.001 keeps the memory negligible, so acc = m + g has the scale of the gradients
+    paths = p.run_and_compare(base, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.001, w.lr, tag="stationary")
+    assert paths[0] == binding.PATH_SAMPLED and all(x == binding.PATH_HINTED for x in paths[1:]), paths
+    paths = p.run_and_compare(base, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.001, w.lr,
+                              use_hint=False, tag="no-hint")
+    assert paths == [binding.PATH_SAMPLED] * 6
+    scales = [1.0, 1.0, 1e-3, 1e-3, 50.0, 50.0]
+    jumpy = [[g * sc for g in step] for step, sc in zip(base, scales)]
+    paths = p.run_and_compare(jumpy, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.001, w.lr, tag="jumps")
+    assert paths == [0, 2, 0, 2, 0, 2], paths
