@@ -348,8 +348,8 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
 #pragma unroll
                 for (int u = 0; u < TK_UNROLL; ++u) {
                     const uint32_t p = pbase + u * (nblocks * TK_UNIT);
-                    const float4 a = __ldcs(reinterpret_cast<const float4*>(P.g + p));
-                    const float4 b = __ldcs(reinterpret_cast<const float4*>(P.m + p));
+                    const float4 a = *reinterpret_cast<const float4*>(P.g + p);
+                    const float4 b = *reinterpret_cast<const float4*>(P.m + p);
                     gv[u][0] = a.x; gv[u][1] = a.y; gv[u][2] = a.z; gv[u][3] = a.w;
                     mv[u][0] = b.x; mv[u][1] = b.y; mv[u][2] = b.z; mv[u][3] = b.w;
                 }
