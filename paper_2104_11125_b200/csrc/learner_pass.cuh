@@ -45,72 +45,87 @@ struct LearnerParams {
 #endif
 };
 
-template <int N, bool VEC>
+// One burst of a thread covers LP_T consecutive tiles x LP_L learners (LP_T * LP_L = LP_UNROLL pairs of
+// 128-bit loads in flight).  Few learners: more tiles per burst keep the loads in flight; many
+// learners: fewer arrays per burst keep each burst inside a few pages.
+template <int N, bool VEC, int LP_T, int LP_L>
 __global__ void __launch_bounds__(LP_THREADS, LP_BLOCKS_PER_SM)
 learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P) {
+    static_assert(LP_T * LP_L == LP_UNROLL, "burst shape");
     const uint32_t tid = threadIdx.x, lane = lane_id();
     const uint32_t d = P.d;
     const int n = P.n;
-    const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside the tile
+    const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside a tile
     const uint32_t sh = (tid & 7u) * 4u;           // and its first bit inside that word
 #ifdef SC_PROFILE_SPANS
     SC_SPAN_BEGIN(P.spans);
 #endif
 
-    for (uint32_t tile = blockIdx.x; tile < P.ntiles; tile += gridDim.x) {
-        // selection bits of this thread's four coordinates and the rank of the first selected one
-        const uint32_t w = __ldg(&P.bitmap[size_t(tile) * 32 + lane]);
-        const uint32_t cnt = __popc(w);
-        const uint32_t incl = warp_incl_scan(cnt);
-        const uint32_t excl_word = __shfl_sync(FULL, incl - cnt, wi);
-        const uint32_t myword = __shfl_sync(FULL, w, wi);
-        const uint32_t nib = (myword >> sh) & 15u;
-        const uint32_t rank0 = __ldg(&P.tile_prefix[tile]) + excl_word + __popc(myword & ((1u << sh) - 1u));
-
-        const uint32_t p = tile * TILE + tid * 4u;
-        if (p >= d) continue;
-
-        float sum[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int i0 = 0; i0 < n; i0 += LP_UNROLL) {
-            float gv[LP_UNROLL][4], mv[LP_UNROLL][4];
+    const uint32_t nsuper = (P.ntiles + LP_T - 1) / LP_T;
+    for (uint32_t sup = blockIdx.x; sup < nsuper; sup += gridDim.x) {
+        // per tile: selection bits of this thread's four coordinates and the rank of the first selected one
+        uint32_t nib[LP_T], rank0[LP_T], pc[LP_T];
 #pragma unroll
-            for (int u = 0; u < LP_UNROLL; ++u)
-                if (i0 + u < n) {
-                    load_quad_stream<VEC>(tab.g[i0 + u], p, d, gv[u]);
-                    load_quad_stream<VEC>(tab.m[i0 + u], p, d, mv[u]);
-                }
-#pragma unroll
-            for (int u = 0; u < LP_UNROLL; ++u)
-                if (i0 + u < n) {
-                    const int i = i0 + u;
-                    float acc[4], out[4];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        acc[c] = __fadd_rn(mv[u][c], gv[u][c]);                        // line 6: m + g
-                        sum[c] = (i == 0) ? acc[c] : __fadd_rn(sum[c], acc[c]);       // line 10, learner order
-                        const float r = ((nib >> c) & 1u) ? 0.0f : acc[c];            // acc - CLT-k(acc)
-                        out[c] = __fadd_rn(__fmul_rn(P.omb, mv[u][c]), __fmul_rn(P.beta, r));   // Eq. 4
-                    }
-                    store_quad_stream<VEC>(tab.m[i], p, d, out);
-                    if (nib && P.gathered) {                                           // Eq. 3: learner i's kept values
-                        uint32_t r = rank0;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            if ((nib >> c) & 1u) P.gathered[size_t(i) * P.k + r++] = acc[c];
-                    }
-                }
+        for (int t = 0; t < LP_T; ++t) {
+            const uint32_t tile = sup * LP_T + t;
+            const bool have = tile < P.ntiles;                         // uniform across the block
+            const uint32_t w = have ? __ldg(&P.bitmap[size_t(tile) * 32 + lane]) : 0u;
+            const uint32_t cnt = __popc(w);
+            const uint32_t incl = warp_incl_scan(cnt);
+            const uint32_t excl_word = __shfl_sync(FULL, incl - cnt, wi);
+            const uint32_t myword = __shfl_sync(FULL, w, wi);
+            nib[t] = (myword >> sh) & 15u;
+            rank0[t] = (have ? __ldg(&P.tile_prefix[tile]) : 0u) + excl_word + __popc(myword & ((1u << sh) - 1u));
+            pc[t] = have ? tile * TILE + tid * 4u : d;                 // d: nothing to do
         }
-        if (nib) {
-            uint32_t r = rank0;
+
+        float sum[LP_T][4];
+        for (int i0 = 0; i0 < n; i0 += LP_L) {
+            float gv[LP_T][LP_L][4], mv[LP_T][LP_L][4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if ((nib >> c) & 1u) {
-                    const float v = __fdiv_rn(sum[c], P.nf);                           // line 10: one division by n
-                    P.out_idx[r] = int32_t(p + c);
-                    P.out_val[r++] = v;
-                    if (P.weights) P.weights[p + c] = __fsub_rn(P.weights[p + c], __fmul_rn(P.lr, v));   // line 12
-                }
+            for (int t = 0; t < LP_T; ++t)
+#pragma unroll
+                for (int u = 0; u < LP_L; ++u)
+                    if (i0 + u < n && pc[t] < d) {
+                        load_quad_stream<VEC>(tab.g[i0 + u], pc[t], d, gv[t][u]);
+                        load_quad_stream<VEC>(tab.m[i0 + u], pc[t], d, mv[t][u]);
+                    }
+#pragma unroll
+            for (int t = 0; t < LP_T; ++t)
+#pragma unroll
+                for (int u = 0; u < LP_L; ++u)
+                    if (i0 + u < n && pc[t] < d) {
+                        const int i = i0 + u;
+                        float acc[4], out[4];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            acc[c] = __fadd_rn(mv[t][u][c], gv[t][u][c]);                    // line 6: m + g
+                            sum[t][c] = (i == 0) ? acc[c] : __fadd_rn(sum[t][c], acc[c]);    // line 10, learner order
+                            const float r = ((nib[t] >> c) & 1u) ? 0.0f : acc[c];            // acc - CLT-k(acc)
+                            out[c] = __fadd_rn(__fmul_rn(P.omb, mv[t][u][c]), __fmul_rn(P.beta, r));   // Eq. 4
+                        }
+                        store_quad_stream<VEC>(tab.m[i], pc[t], d, out);
+                        if (nib[t] && P.gathered) {                                           // Eq. 3: learner i's kept values
+                            uint32_t r = rank0[t];
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                if ((nib[t] >> c) & 1u) P.gathered[size_t(i) * P.k + r++] = acc[c];
+                        }
+                    }
         }
+#pragma unroll
+        for (int t = 0; t < LP_T; ++t)
+            if (nib[t] && pc[t] < d) {
+                uint32_t r = rank0[t];
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if ((nib[t] >> c) & 1u) {
+                        const float v = __fdiv_rn(sum[t][c], P.nf);                           // line 10: one division by n
+                        P.out_idx[r] = int32_t(pc[t] + c);
+                        P.out_val[r++] = v;
+                        if (P.weights) P.weights[pc[t] + c] = __fsub_rn(P.weights[pc[t] + c], __fmul_rn(P.lr, v));   // line 12
+                    }
+            }
     }
 #ifdef SC_PROFILE_SPANS
     SC_SPAN_END(P.spans);

@@ -35,6 +35,7 @@ struct scalecom_ctx {
     // launch geometry
     int sms = 0;
     uint32_t topk_blocks = 0, lp_blocks = 0;
+    int lp_tiles = 1;                  // tiles per burst of the learner pass
     uint32_t samp_stride = 1, samp_target = 1;
 
     // options
@@ -85,22 +86,35 @@ cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
                                        dim3(TK_THREADS), args, sizeof(TopkShared), c->stream);
 }
 
-template <int N, bool VEC>
+template <int N, bool VEC, int T>
 cudaError_t launch_learner(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
     PtrTable<N> tab;
     for (int i = 0; i < N; ++i) {
         tab.g[i] = i < c->n ? grads[i] : nullptr;
         tab.m[i] = i < c->n ? mem[i] : nullptr;
     }
-    learner_pass_kernel<N, VEC><<<c->lp_blocks, LP_THREADS, 0, c->stream>>>(tab, P);
+    const uint32_t nsuper = (c->ntiles + T - 1) / T;
+    const uint32_t blocks = c->lp_blocks < nsuper ? c->lp_blocks : nsuper;
+    learner_pass_kernel<N, VEC, T, LP_UNROLL / T><<<blocks, LP_THREADS, 0, c->stream>>>(tab, P);
     return cudaGetLastError();
+}
+
+// burst shape (tiles x learners) by learner count
+template <int N, bool VEC>
+cudaError_t launch_learner_t(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
+    switch (c->lp_tiles) {
+        case 1: return launch_learner<N, VEC, 1>(c, grads, mem, P);
+        case 2: return launch_learner<N, VEC, 2>(c, grads, mem, P);
+        case 4: return launch_learner<N, VEC, 4>(c, grads, mem, P);
+        default: return launch_learner<N, VEC, 8>(c, grads, mem, P);
+    }
 }
 
 template <bool VEC>
 cudaError_t launch_learner_n(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
-    if (c->n <= 16) return launch_learner<16, VEC>(c, grads, mem, P);
-    if (c->n <= 128) return launch_learner<128, VEC>(c, grads, mem, P);
-    return launch_learner<SCALECOM_MAX_LEARNERS, VEC>(c, grads, mem, P);
+    if (c->n <= 16) return launch_learner_t<16, VEC>(c, grads, mem, P);
+    if (c->n <= 128) return launch_learner_t<128, VEC>(c, grads, mem, P);
+    return launch_learner_t<SCALECOM_MAX_LEARNERS, VEC>(c, grads, mem, P);
 }
 
 int init_workspace(scalecom_ctx* c) {
@@ -245,7 +259,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
         if (o2 < occ_topk) occ_topk = o2;
     }
     if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_lp, learner_pass_kernel<16, true>, LP_THREADS, 0);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_lp, learner_pass_kernel<16, true, 1, LP_UNROLL>, LP_THREADS, 0);
     if (e != cudaSuccess || !coop || occ_topk < 1 || occ_lp < 1) {
         cudaGetLastError();
         delete c;
@@ -262,6 +276,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->tiles_per_block = (c->ntiles + c->topk_blocks - 1) / c->topk_blocks;
     c->lp_blocks = uint32_t(c->sms * occ_lp);
     if (c->lp_blocks > c->ntiles) c->lp_blocks = c->ntiles;
+    c->lp_tiles = n >= 8 ? 1 : n >= 4 ? 2 : n >= 2 ? 4 : 8;
 
     // sampling rate: about 2^18 sampled keys or 1/64 of the vector, whichever is more
     uint32_t stride = 1;
