@@ -13,7 +13,9 @@ enumeration on tiny d (Eq. 2), k = d reducing to dense averaged SGD
 error-feedback top-k (Remark 1), acc = sparse + residual (Eq. 4), leader
 cycling (Algorithm 1 line 6), commutativity (Eq. 1), the virtual-sequence
 identity of Appendix D.1, the contraction identity of Appendix C and a
-library top-k cross-check.  No function here is "parity unpinned".
+library top-k cross-check; the chunk-wise selector by per-chunk brute force,
+its k = d and k = 1 limits and the structure of Appendix E's demonstration.
+No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -54,6 +56,9 @@ def _load():
         for sfx, real in (("f32", ctypes.c_float), ("f64", ctypes.c_double)):
             f = getattr(_lib, "oracle_rank_" + sfx); f.restype = i64; f.argtypes = [vp, i64, i64]
             f = getattr(_lib, "oracle_topk_" + sfx); f.restype = ctypes.c_int; f.argtypes = [vp, i64, i64, vp, vp]
+            f = getattr(_lib, "oracle_chunk_select_" + sfx); f.restype = ctypes.c_int; f.argtypes = [vp, i64, i64, vp, vp]
+            f = getattr(_lib, "oracle_step_sel_" + sfx); f.restype = ctypes.c_int
+            f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, ctypes.c_int, vp, vp, vp]
             f = getattr(_lib, "oracle_accumulate_" + sfx); f.restype = None; f.argtypes = [vp, vp, i64, vp]
             f = getattr(_lib, "oracle_learner_" + sfx); f.restype = None
             f.argtypes = [vp, vp, i64, vp, i64, vp, real, vp]
@@ -103,6 +108,20 @@ def topk(x: np.ndarray, k: int):
     return idx, sel
 
 
+SELECTORS = {"topk": 0, "chunk": 1}
+
+
+def chunk_select(x: np.ndarray, k: int):
+    """Chunk-wise selection (Section 4 / Appendix E): one coordinate from each of k consecutive
+    chunks; returns (idx int32[k] ascending, sel uint8[d])."""
+    lib = _load()
+    d = x.size
+    idx = np.empty(k, np.int32)
+    sel = np.empty(d, np.uint8)
+    getattr(lib, "oracle_chunk_select_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), d, int(k), _p(idx), _p(sel))
+    return idx, sel
+
+
 def accumulate(g: np.ndarray, m: np.ndarray) -> np.ndarray:
     """acc = m + g (the argument of CLT-k, Algorithm 1 line 6)."""
     lib = _load()
@@ -137,8 +156,9 @@ def apply(theta: np.ndarray, idx: np.ndarray, val: np.ndarray, lr: float) -> Non
     getattr(lib, "oracle_apply_" + _sfx(theta.dtype))(_p(_chk(theta, theta.dtype)), _p(idx), _p(val), idx.size, float(lr))
 
 
-def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: bool = True):
-    """One iteration of Algorithm 1.
+def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: bool = True,
+         selector: str = "topk"):
+    """One iteration of Algorithm 1 ("topk": Eq. 2 on the leader; "chunk": chunk-wise selection).
 
     g, m: lists of n ndarrays of d values (m updated in place); theta: ndarray
     of d values updated in place, or None.  Returns (idx, val, G) with G the
@@ -157,10 +177,11 @@ def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: boo
     idx = np.empty(k, np.int32)
     val = np.empty(k, dtype)
     G = np.empty((n, k), dtype) if want_gathered else None
-    rc = getattr(lib, "oracle_step_" + _sfx(dtype))(
+    rc = getattr(lib, "oracle_step_sel_" + _sfx(dtype))(
         ctypes.cast(gp, ctypes.c_void_p), ctypes.cast(mp, ctypes.c_void_p),
         _p(theta) if theta is not None else None,
-        int(t), n, d, int(k), float(beta), float(lr), _p(idx), _p(val), _p(G) if G is not None else None)
+        int(t), n, d, int(k), float(beta), float(lr), SELECTORS[selector], _p(idx), _p(val),
+        _p(G) if G is not None else None)
     if rc != 0:
         raise MemoryError("oracle_step")
     return idx, val, G

@@ -299,3 +299,60 @@ def test_pieces_compose_to_step():
     oracle.apply(th2, idx2, val2, lr)
     assert np.array_equal(idx, idx2) and np.array_equal(val, val2) and np.array_equal(G, G2)
     assert all(np.array_equal(a, b) for a, b in zip(m1, m2)) and np.array_equal(th1, th2)
+
+
+# ---- chunk-wise selector (Section 4, Appendix E) -----------------------------------------------
+def test_chunk_select_brute_force_and_limits():
+    for x in tie_vectors():
+        d = x.size
+        key = key32(x).astype(np.int64)
+        for k in range(1, d + 1):
+            idx, sel = oracle.chunk_select(x, k)
+            bounds = [(j * d) // k for j in range(k + 1)]
+            assert bounds[0] == 0 and bounds[-1] == d and all(b > a for a, b in zip(bounds, bounds[1:]))
+            expect = []
+            for j in range(k):
+                chunk = range(bounds[j], bounds[j + 1])
+                best = max(chunk, key=lambda p: (key[p], -p))         # largest magnitude, then lowest index
+                expect.append(best)
+            assert idx.tolist() == expect
+            assert sel.tolist() == [1 if p in expect else 0 for p in range(d)]
+            assert np.array_equal(oracle.chunk_select(x.astype(np.float64), k)[0], idx)
+        assert oracle.chunk_select(x, d)[0].tolist() == list(range(d))          # k = d keeps everything
+        assert oracle.chunk_select(x, 1)[0].tolist() == oracle.topk(x, 1)[0].tolist()   # k = 1 is the top-1 set
+
+
+def test_chunk_select_matches_the_demonstration_structure():
+    path = os.path.join(os.path.dirname(__file__), "golden", "chunk_demo.txt")
+    row = [l for l in open(path) if l.strip() and not l.startswith("#")][0].split()
+    d, k = int(row[0]), int(row[1])
+    chunk_of = list(map(int, row[2:2 + d]))
+    picks = list(map(int, row[2 + d:2 + d + k]))
+    x = np.full(d, 0.1, np.float32)
+    for j, local in enumerate(picks):                      # make the demonstrated local index the chunk's largest
+        x[chunk_of.index(j) + local] = -3.0 - j
+    idx, sel = oracle.chunk_select(x, k)
+    assert [chunk_of[p] for p in idx] == list(range(k))
+    assert [p - chunk_of.index(j) for j, p in enumerate(idx)] == picks
+
+
+def test_chunk_step_is_the_same_algorithm_with_another_index_set():
+    n, d, k, beta, lr, t = 3, 1000, 37, 0.1, 0.05, 5
+    g = [RNG.standard_normal(d) for _ in range(n)]
+    m = [RNG.standard_normal(d) for _ in range(n)]
+    th = RNG.standard_normal(d)
+    m1, th1 = [a.copy() for a in m], th.copy()
+    idx, val, G = oracle.step(g, m1, th1, t, k, beta, lr, selector="chunk")
+    acc = np.stack([a + b for a, b in zip(m, g)])
+    assert np.array_equal(idx, oracle.chunk_select(acc[t % n].copy(), k)[0])
+    np.testing.assert_allclose(val, acc[:, idx].mean(axis=0), rtol=1e-13)          # Eq. 1 with the chunk set
+    np.testing.assert_array_equal(G, acc[:, idx])
+    for i in range(n):
+        r = acc[i].copy(); r[idx] = 0.0
+        np.testing.assert_allclose(m1[i], (1 - beta) * m[i] + beta * r, rtol=1e-13, atol=1e-15)   # Eq. 4
+    expect = th.copy(); expect[idx] -= lr * val
+    np.testing.assert_allclose(th1, expect, rtol=1e-14)
+    # contraction of any index set of size k (proof of Lemma 1): ||x - comp(x)||^2 = ||x||^2 - sum over the set
+    x = acc[t % n]
+    comp = np.zeros(d); comp[idx] = x[idx]
+    np.testing.assert_allclose(np.sum((x - comp) ** 2), np.sum(x ** 2) - np.sum(x[idx] ** 2), rtol=1e-12)
