@@ -43,6 +43,8 @@ def parse_args():
     ap.add_argument("--batches", type=int, default=MAX_BATCHES,
                     help="distinct gradient batches kept in HBM (steps cycle through them); small values keep "
                          "the footprint low for profiler captures")
+    ap.add_argument("--selector", default="topk", choices=["topk", "chunk"],
+                    help="leader selection: exact top-k (the headline path) or the chunk-wise selector")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -157,11 +159,11 @@ def run_reference(args):
     th = W.initial_weights(w, "cpu").numpy()
     t = 0
     for _ in range(args.warmup):
-        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False)
+        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False, selector=args.selector)
         t += 1
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False)
+        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False, selector=args.selector)
         t += 1
     dt = time.perf_counter() - t0
     value = w.n * w.d * args.steps / dt
@@ -178,7 +180,7 @@ def run_reference(args):
     }))
 
 
-def time_oracle(w, batches_dev, steps=2):
+def time_oracle(w, batches_dev, steps=2, selector="topk"):
     """cpu_baseline leg: the oracle on full-size steps of the bench workload, on this machine's host cores."""
     import numpy as np
     import oracle
@@ -188,7 +190,7 @@ def time_oracle(w, batches_dev, steps=2):
     for s in range(steps):
         g = [x.cpu().numpy() for x in batches_dev[s % len(batches_dev)]]
         t0 = time.perf_counter()
-        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False)
+        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False, selector=selector)
         dt += time.perf_counter() - t0
     return {"value": w.n * w.d * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
             "sample": "%d full steps of the bench workload (n=%d, d=%d, k=%d), %.1f s" % (steps, w.n, w.d, w.k, dt)}
@@ -232,6 +234,8 @@ def main():
 
     stream = torch.cuda.Stream(device=dev)
     ctx = sc.Context(w.d, w.n, w.k, w.beta, w.lr, stream=stream)
+    if args.selector == "chunk":
+        ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK)
     torch.cuda.synchronize()
 
     # ---- device-resident timing ---------------------------------------------------------------------
@@ -314,7 +318,8 @@ def main():
             "config": {"workload": w.name, "n": w.n, "d": w.d, "k": w.k, "beta": w.beta, "lr": w.lr,
                        "parallelism": "replicas only" if world > 1 else "single GPU, n logical learners",
                        "l2": "inputs larger than L2 (%.2f GB of g+m per step), no flush" % (8e-9 * w.n * w.d),
-                       "gradient_batches_resident": nb, "selection_path_last_step": paths,
+                       "gradient_batches_resident": nb, "selector": args.selector,
+                       "selection_path_last_step": paths,
                        "weight_update": "fused into the learner pass"},
             "roofline": {"bound": "hbm", "kernel": "learner_pass_kernel", "achieved": lp_gbs, "peak": peak,
                          "unit": "GB/s", "frac": lp_gbs / peak, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
@@ -332,7 +337,7 @@ def main():
                           "h2d_bytes_per_step": 4 * w.n * w.d, "d2h_bytes_per_step": 8 * w.k,
                           "ms_per_step": e2e_ms, "api": "scalecom_step_host (pinned host gradients in, idx/val out)"}
         if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = time_oracle(w, batches)
+            out["cpu_baseline"] = time_oracle(w, batches, selector=args.selector)
         print(json.dumps(out))
     ctx.close()
     if world > 1:

@@ -148,12 +148,22 @@ int scalecom_reset(scalecom_ctx* ctx);
 #define SCALECOM_OPT_USE_HINT         5  /* 1 (default): a step starts its pre-filter from the threshold the
                                             previous step of this handle found; 0: always sample afresh.
                                             Affects speed only, never results                              */
+#define SCALECOM_OPT_SELECTOR         6  /* how the leader's index set is found (results DO differ):
+                                            SCALECOM_SELECTOR_TOPK (default): the exact top-k set of Eq. 2;
+                                            SCALECOM_SELECTOR_CHUNK: the chunk-wise selection of Section 4 /
+                                            Appendix E -- the d coordinates form k consecutive chunks,
+                                            chunk j = [floor(j*d/k), floor((j+1)*d/k)), and each keeps its
+                                            largest-magnitude coordinate (lower index on ties).  Steps 1, 3,
+                                            4, 5 are unchanged.  First use allocates 8*k bytes             */
+#define SCALECOM_SELECTOR_TOPK  0
+#define SCALECOM_SELECTOR_CHUNK 1
 int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 
 /* Items for scalecom_query (each synchronises the stream when it reads device state). */
 #define SCALECOM_Q_WORKSPACE_BYTES  1  /* device bytes owned by the handle                                    */
 #define SCALECOM_Q_LAST_TOPK_PATH   2  /* last step's selection path: 0 = sampled pre-filter, 1 = full select,
-                                          2 = pre-filter started from the previous step's threshold           */
+                                          2 = pre-filter started from the previous step's threshold,
+                                          3 = chunk-wise selector                                             */
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */

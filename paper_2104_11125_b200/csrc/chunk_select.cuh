@@ -1,0 +1,171 @@
+// Chunk-wise leader selection (Section 4: the buffer is cut into chunks that are searched
+// independently; Appendix E's demonstration keeps one index per chunk).
+//
+// The d coordinates form k consecutive chunks, chunk j = [floor(j*d/k), floor((j+1)*d/k)); each
+// contributes the coordinate of acc = m + g that comes first in the order "larger |acc| first,
+// lower index first".  One streaming read of g and m, one grid barrier:
+//   S1  stream: one warp per chunk (lanes read the chunk in coalesced rows of 32), a hardware warp
+//       max finds the largest key, a warp min the lowest index holding it; the owner stores the
+//       composite (key << 31) | (2^31 - 1 - idx) in best[j]
+//   S2  after the barrier: thread j turns best[j] into the bitmap bit and the index list entry;
+//       a tile's prefix count needs no scan -- exactly one coordinate is kept per chunk, so the
+//       count before coordinate p0 is the number of chunks before p0's chunk, plus one if that
+//       chunk's pick lies before p0
+#pragma once
+#include "common.cuh"
+
+namespace sc {
+
+#ifndef SC_CS_THREADS
+#define SC_CS_THREADS 512
+#endif
+#ifndef SC_CS_BLOCKS_PER_SM
+#define SC_CS_BLOCKS_PER_SM 3
+#endif
+constexpr int CS_THREADS = SC_CS_THREADS;
+constexpr int CS_BLOCKS_PER_SM = SC_CS_BLOCKS_PER_SM;
+#ifndef SC_CS_GROUP
+#define SC_CS_GROUP 2
+#endif
+constexpr int CS_GROUP = SC_CS_GROUP;           // chunks a warp works on at a time
+constexpr int CS_UNROLL = 4;                    // rows of 32 coordinates of each of them in flight
+
+struct ChunkParams {
+    const float* g;
+    const float* m;
+    uint32_t d, k;
+    double inv_d;                       // 1.0 / d
+    uint32_t spin_limit;
+    unsigned long long* best;           // [k] composite of every chunk's pick, rewritten by every launch
+    uint32_t* bitmap;                   // [ntiles * 32]
+    uint32_t* tile_prefix;              // [ntiles + 1]
+    uint32_t ntiles;
+    uint32_t* ctrl;                     // status word at [CT_STATUS], path at [CT_PATH]
+    unsigned long long* barrier;        // arrival counter used by this kernel only
+    int32_t* out_idx;                   // [k] or nullptr
+#ifdef SC_PROFILE_SPANS
+    unsigned long long* spans;
+#endif
+};
+
+// Chunk of coordinate p: the j with j*d < (p+1)*k <= (j+1)*d.
+__device__ __forceinline__ uint32_t chunk_of(uint32_t p, uint32_t d, uint32_t k, double inv_d) {
+    const uint64_t x = (uint64_t(p) + 1u) * k;
+    uint64_t j = uint64_t(__double2ull_rd(double(x - 1u) * inv_d));       // within one of the answer
+    if (j * d >= x) --j;
+    else if ((j + 1u) * d < x) ++j;
+    return uint32_t(j);
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(CS_THREADS, CS_BLOCKS_PER_SM) chunk_select_kernel(const ChunkParams P) {
+    __shared__ int flag;
+    const uint32_t tid = threadIdx.x, lane = lane_id();
+    const uint32_t nblocks = gridDim.x;
+    const size_t gtid = size_t(blockIdx.x) * CS_THREADS + tid;
+    const size_t gsize = size_t(nblocks) * CS_THREADS;
+    const uint32_t d = P.d, k = P.k;
+    GridBarrier gb;
+    gb.arrive = P.barrier; gb.nblocks = nblocks; gb.status = P.ctrl + 1; gb.spin_limit = P.spin_limit;
+    SC_SPAN_BEGIN(P.spans);
+
+    // the bitmap is first written after the barrier
+    {
+        const size_t nv = size_t(P.ntiles) * 8;
+        uint4* pv = reinterpret_cast<uint4*>(P.bitmap);
+        for (size_t i = gtid; i < nv; i += gsize) pv[i] = make_uint4(0, 0, 0, 0);
+    }
+
+    // ---------------- S1: one warp per chunk, chunks dealt round-robin to the warps of the grid --------
+    // Lane i reads elements lo + i, lo + i + 32, ... of the chunk (coalesced 128-byte rows; a chunk
+    // need not start on a 16-byte boundary), keeps its best, and one hardware warp max plus a ballot
+    // pick the chunk's winner.  Every chunk has one owner: plain stores, no atomics.
+    // Chunk bounds without a division per chunk: j*d = q*k + r is carried along as j advances.
+    const uint32_t warps = nblocks * (CS_THREADS / 32);
+    const uint32_t gw = blockIdx.x * (CS_THREADS / 32) + (tid >> 5);
+    const uint32_t dq = d / k, dr = d % k;                              // d = dq*k + dr
+    const uint64_t sd = uint64_t(warps) * CS_GROUP * d;                 // a warp advances by warps*CS_GROUP chunks
+    const uint32_t sq = uint32_t(sd / k), sr = uint32_t(sd % k);        // sd = sq*k + sr
+    const uint64_t j0 = uint64_t(gw) * CS_GROUP;
+    uint32_t q = uint32_t(j0 * d / k), r = uint32_t(j0 * d % k);        // j*d = q*k + r for the group's first chunk
+    for (uint64_t j = j0; j < k; j += uint64_t(warps) * CS_GROUP) {
+        // bounds of the group's chunks: lo[g] = floor((j+g)*d/k), chained without divisions
+        uint32_t lo[CS_GROUP + 1];
+        {
+            uint32_t qq = q, rr = r;
+            lo[0] = qq;
+#pragma unroll
+            for (int g = 1; g <= CS_GROUP; ++g) {
+                qq += dq; rr += dr;                                     // rr, dr < k <= 2^31: no overflow
+                if (rr >= k) { rr -= k; ++qq; }
+                lo[g] = (j + g <= k) ? qq : lo[g - 1];                  // chunks past the last one are empty
+            }
+        }
+        uint32_t bk[CS_GROUP], bi[CS_GROUP];                            // this lane's best key and its index, per chunk
+        bool have[CS_GROUP];
+#pragma unroll
+        for (int g = 0; g < CS_GROUP; ++g) { bk[g] = 0; bi[g] = 0xFFFFFFFFu; have[g] = false; }
+        // rows of 32 coordinates, CS_UNROLL rows of every chunk of the group in flight at a time
+        uint32_t longest = 0;
+#pragma unroll
+        for (int g = 0; g < CS_GROUP; ++g) longest = max(longest, lo[g + 1] - lo[g]);
+        for (uint32_t off = 0; off < longest; off += 32u * CS_UNROLL) {
+            float gv[CS_GROUP][CS_UNROLL], mv[CS_GROUP][CS_UNROLL];
+#pragma unroll
+            for (int g = 0; g < CS_GROUP; ++g)
+#pragma unroll
+                for (int u = 0; u < CS_UNROLL; ++u) {
+                    const uint32_t p = lo[g] + off + u * 32u + lane;
+                    if (p < lo[g + 1]) { gv[g][u] = P.g[p]; mv[g][u] = P.m[p]; }
+                }
+#pragma unroll
+            for (int g = 0; g < CS_GROUP; ++g)
+#pragma unroll
+                for (int u = 0; u < CS_UNROLL; ++u) {
+                    const uint32_t p = lo[g] + off + u * 32u + lane;
+                    if (p < lo[g + 1]) {
+                        const uint32_t key = mag_key(__fadd_rn(mv[g][u], gv[g][u]));
+                        if (!have[g] || key > bk[g]) { bk[g] = key; bi[g] = p; have[g] = true; }   // strict: lower index stays on ties
+                    }
+                }
+        }
+#pragma unroll
+        for (int g = 0; g < CS_GROUP; ++g) {
+            if (j + g >= k) break;                                      // warp-uniform
+            const uint32_t mx = __reduce_max_sync(FULL, have[g] ? bk[g] : 0u);
+            // among lanes holding the maximum, the lowest index wins
+            const uint32_t best_idx = __reduce_min_sync(FULL, (have[g] && bk[g] == mx) ? bi[g] : 0xFFFFFFFFu);
+            if (lane == 0) P.best[j + g] = composite(mx, best_idx);
+        }
+        q += sq; r += sr;
+        if (r >= k) { r -= k; ++q; }
+    }
+    if (!grid_barrier(gb, &flag)) return;
+
+    // ---------------- S2: bitmap, index list, tile prefixes ----------------------------------------
+    for (size_t jj = gtid; jj < k; jj += gsize) {
+        const unsigned long long b = __ldcg(&P.best[jj]);
+        const uint32_t idx = 0x7FFFFFFFu - uint32_t(b & 0x7FFFFFFFull);
+        if (b == 0ull || idx >= d) {                                    // every chunk holds at least one coordinate
+            atomicCAS(P.ctrl + 1, DEV_OK, DEV_INTERNAL);
+        } else {
+            atomicOr(&P.bitmap[idx >> 5], 1u << (idx & 31u));
+            if (P.out_idx) P.out_idx[jj] = int32_t(idx);
+        }
+    }
+    for (size_t tile = gtid; tile <= P.ntiles; tile += gsize) {
+        uint32_t prefix = k;                                            // the sentinel entry at ntiles
+        if (tile < P.ntiles) {
+            const uint32_t p0 = uint32_t(tile) * TILE;                  // < d
+            const uint32_t jt = chunk_of(p0, d, k, P.inv_d);
+            const unsigned long long b = __ldcg(&P.best[jt]);
+            const uint32_t idx = 0x7FFFFFFFu - uint32_t(b & 0x7FFFFFFFull);
+            prefix = jt + (idx < p0 ? 1u : 0u);
+        }
+        P.tile_prefix[tile] = prefix;
+    }
+    if (gtid == 0) { P.ctrl[2] = 3u; P.ctrl[3] = k; }                   // path 3: chunk-wise; "candidates" = k
+    SC_SPAN_END(P.spans);
+}
+
+}  // namespace sc

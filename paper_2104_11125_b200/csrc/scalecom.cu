@@ -9,6 +9,7 @@
 #include <cstring>
 #include <new>
 
+#include "chunk_select.cuh"
 #include "learner_pass.cuh"
 #include "topk_select.cuh"
 
@@ -41,6 +42,9 @@ struct scalecom_ctx {
     // options
     uint32_t force_exact = 0;
     uint32_t use_hint = 1;
+    int selector = SCALECOM_SELECTOR_TOPK;
+    unsigned long long* chunk_best = nullptr;   // [k], allocated when the chunk-wise selector is first chosen
+    uint32_t chunk_blocks = 0;
     uint32_t spin_limit = 1u << 22;
     bool timing = false;
     bool fuse_update = true;
@@ -86,6 +90,13 @@ cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
                                        dim3(TK_THREADS), args, sizeof(TopkShared), c->stream);
 }
 
+template <bool VEC>
+cudaError_t launch_chunk(const scalecom_ctx* c, const ChunkParams& P) {
+    void* args[] = {const_cast<ChunkParams*>(&P)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&chunk_select_kernel<VEC>), dim3(c->chunk_blocks),
+                                       dim3(CS_THREADS), args, 0, c->stream);
+}
+
 template <int N, bool VEC, int T>
 cudaError_t launch_learner(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
     PtrTable<N> tab;
@@ -119,6 +130,8 @@ cudaError_t launch_learner_n(const scalecom_ctx* c, const float* const* grads, f
 
 int init_workspace(scalecom_ctx* c) {
     if (cudaMemsetAsync(c->ws, 0, c->ctrl_region_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (c->chunk_best && cudaMemsetAsync(c->chunk_best, 0, size_t(c->k) * 8, c->stream) != cudaSuccess)
+        return SCALECOM_ERR_CUDA;
     return SCALECOM_OK;
 }
 
@@ -205,7 +218,24 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     const bool tm = c->timing && c->ev;
     cudaEvent_t* ev = tm ? c->ev + 4 * (c->ev_steps % scalecom_ctx::EV_RING) : nullptr;
     if (tm && cudaEventRecord(ev[0], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
-    cudaError_t e = vec_leader ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
+    cudaError_t e;
+    if (c->selector == SCALECOM_SELECTOR_CHUNK) {
+        ChunkParams cp;
+        cp.g = tp.g; cp.m = tp.m; cp.d = tp.d; cp.k = tp.k;
+        cp.inv_d = 1.0 / double(c->d);
+        cp.spin_limit = c->spin_limit;
+        cp.best = c->chunk_best;
+        cp.bitmap = c->bitmap; cp.tile_prefix = c->tile_prefix; cp.ntiles = c->ntiles;
+        cp.ctrl = c->ctrl;
+        cp.barrier = c->barrier + 8;               // its own arrival counter: the grid differs from the top-k kernel's
+        cp.out_idx = nullptr;                      // written by the learner pass
+#ifdef SC_PROFILE_SPANS
+        cp.spans = c->spans;
+#endif
+        e = vec_leader ? launch_chunk<true>(c, cp) : launch_chunk<false>(c, cp);
+    } else {
+        e = vec_leader ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
+    }
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     if (tm && cudaEventRecord(ev[1], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
@@ -405,6 +435,7 @@ void scalecom_destroy(scalecom_ctx* c) {
         delete[] c->ev;
     }
     cudaFree(c->ws);
+    cudaFree(c->chunk_best);
     cudaFree(c->stage_g);
     cudaFree(c->stage_idx);
     cudaFree(c->stage_val);
@@ -489,6 +520,29 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
         }
         case SCALECOM_OPT_FUSE_UPDATE: c->fuse_update = value != 0; return SCALECOM_OK;
         case SCALECOM_OPT_USE_HINT: c->use_hint = value ? 1u : 0u; return SCALECOM_OK;
+        case SCALECOM_OPT_SELECTOR: {
+            if (value != SCALECOM_SELECTOR_TOPK && value != SCALECOM_SELECTOR_CHUNK) return SCALECOM_ERR_INVALID_ARG;
+            if (value == SCALECOM_SELECTOR_CHUNK && !c->chunk_best) {
+                DeviceGuard guard(c->device);
+                int occ = 0;
+                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, chunk_select_kernel<true>, CS_THREADS, 0) != cudaSuccess ||
+                    occ < 1)
+                    return SCALECOM_ERR_CUDA;
+                if (occ > CS_BLOCKS_PER_SM) occ = CS_BLOCKS_PER_SM;
+                const int64_t per_block = int64_t(CS_THREADS / 32) * CS_GROUP;                 // chunks one block takes per round
+                const uint32_t need = uint32_t((c->k + per_block - 1) / per_block);
+                c->chunk_blocks = uint32_t(c->sms * occ) < need ? uint32_t(c->sms * occ) : need;
+                const size_t bytes = size_t(c->k) * 8;
+                if (cudaMalloc(reinterpret_cast<void**>(&c->chunk_best), bytes) != cudaSuccess) {
+                    cudaGetLastError();
+                    c->chunk_best = nullptr;
+                    return SCALECOM_ERR_ALLOC;
+                }
+                if (cudaMemsetAsync(c->chunk_best, 0, bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+            }
+            c->selector = int(value);
+            return SCALECOM_OK;
+        }
         default: return SCALECOM_ERR_INVALID_ARG;
     }
 }

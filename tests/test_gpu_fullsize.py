@@ -111,3 +111,11 @@ def test_config5_large_windows():
     if free < 110 * 2 ** 30:
         pytest.skip("needs ~105 GB of free device memory")
     fullsize_case(W.LARGE, steps=2)
+
+
+@pytest.mark.parametrize("w", [W.RESNET50, W.TRANSFORMER], ids=lambda w: w.name)
+def test_chunk_selector_full_size_every_element(w):
+    """The chunk-wise oracle needs no sort, so whole steps at full size are compared element by element."""
+    from tests.parity import workload_case
+    paths = workload_case(w, 2, DEV, selector="chunk")
+    assert paths == [3, 3]

@@ -221,3 +221,56 @@ def test_threshold_hint_is_used_then_survives_scale_jumps():
     jumpy = [[g * sc for g in step] for step, sc in zip(base, scales)]
     paths = p.run_and_compare(jumpy, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.001, w.lr, tag="jumps")
     assert paths == [0, 2, 0, 2, 0, 2], paths
+
+
+# ---- chunk-wise selector (Section 4 / Appendix E) ----------------------------------------------------
+@pytest.mark.parametrize("base,d,n,steps", [
+    (W.TINY, 1 << 20, 4, 3),
+    (W.RESNET50, 1_500_013, 8, 3),
+    (W.TRANSFORMER, 2_000_003, 16, 2),
+    (W.RESNET50, 50_001, 130, 2),
+])
+def test_chunk_selector_scaled_workloads(base, d, n, steps):
+    paths = _parity().workload_case(base.scaled(d, n=n), steps, DEV, selector="chunk")
+    assert all(p == 3 for p in paths)
+
+
+def test_chunk_selector_edge_cases():
+    rng = np.random.default_rng(11)
+    kw = dict(selector="chunk")
+    _edge([[3.0]], 1, tag="chunk d=1", **kw)
+    _edge([np.zeros(5000)] * 2, 77, tag="chunk all-zero", **kw)
+    pm = np.where(np.arange(9001) % 2 == 0, 1.0, -1.0)
+    _edge([pm, -pm], 4500, tag="chunk ties", **kw)
+    x = rng.standard_normal(10_007)
+    _edge([x, 0.5 * x], 1, tag="chunk k=1", **kw)
+    _edge([x, 0.5 * x], 10_007, tag="chunk k=d", **kw)
+    _edge([x, 0.5 * x], 5003, tag="chunk of two or three", **kw)
+    _edge([x, 0.5 * x], 3337, tag="chunk of three", **kw)
+    _edge([x], 71, beta=1.0, tag="chunk n=1", **kw)
+    q = rng.integers(-3, 4, 50_000).astype(np.float32)
+    _edge([q, np.roll(q, 1)], 499, tag="chunk quantised", **kw)
+    for off in (1, 3):
+        w = W.TINY.scaled(100_003)
+        _parity().workload_case(w, 2, DEV, offset=off, selector="chunk")
+
+
+def test_switching_selectors_on_one_handle():
+    import paper_2104_11125_b200 as sc
+    import oracle
+    from paper_2104_11125_b200 import binding
+    w = W.TINY.scaled(300_000)
+    prof = W.profile(w, DEV)
+    m = W.initial_memory(w, DEV)
+    m_o = [x.cpu().numpy().copy() for x in m]
+    idx = torch.empty(w.k, device=DEV, dtype=torch.int32)
+    val = torch.empty(w.k, device=DEV)
+    with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
+        for t, sel in enumerate(["topk", "chunk", "chunk", "topk", "chunk", "topk"]):
+            ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK if sel == "chunk" else binding.SELECTOR_TOPK)
+            g = W.gradients(w, t, DEV, prof)
+            ctx.step(g, m, None, t, idx, val)
+            assert ctx.status() == 0
+            idx_o, val_o, _ = oracle.step([x.cpu().numpy() for x in g], m_o, None, t, w.k, w.beta, w.lr, selector=sel)
+            assert np.array_equal(idx.cpu().numpy(), idx_o) and np.array_equal(val.cpu().numpy(), val_o), (t, sel)
+        assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(m, m_o))
