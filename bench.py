@@ -261,6 +261,7 @@ def main():
     ms_total = ev0.elapsed_time(ev1)
     launches = ctx.query(binding.Q_KERNEL_LAUNCHES) - launches0
     ctx.set_option(binding.OPT_KERNEL_TIMING, 1)
+    ctx.set_option(binding.OPT_KERNEL_SPANS, 1)
     evb0, evb1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     evb0.record(stream)
     for _ in range(K):
@@ -272,7 +273,9 @@ def main():
     ms_total_b = evb0.elapsed_time(evb1)
     assert ctx.status() == 0, "device status %d" % ctx.status()
     kms, ksteps = ctx.kernel_ms()
+    sms, ssteps = ctx.kernel_span_ms()
     ctx.set_option(binding.OPT_KERNEL_TIMING, 0)
+    ctx.set_option(binding.OPT_KERNEL_SPANS, 0)
     paths = ctx.query(binding.Q_LAST_TOPK_PATH)
 
     # ---- end to end through the host-buffer entry point ------------------------------------------------
@@ -328,7 +331,13 @@ def main():
                          "topk_select_kernel": {"achieved": tk_gbs, "frac": tk_gbs / peak, "avg_launch_ms": tk_ms,
                                                 "algorithmic_bytes_per_launch": tk_bytes,
                                                 "frac_of_nominal_8TBs": tk_gbs / NOMINAL_HBM_GBS},
-                         "steps_timed": ksteps, "ms_per_step_with_kernel_events": ms_total_b / K},
+                         "steps_timed": ksteps, "ms_per_step_with_kernel_events": ms_total_b / K,
+                         "in_kernel_ms": {"note": "first block start to last block end on the GPU timer, no launch "
+                                                  "gap or event overhead; same steps as the event figures",
+                                          "learner_pass_kernel": sms[1] / max(ssteps, 1),
+                                          "topk_select_kernel": sms[0] / max(ssteps, 1),
+                                          "learner_frac": lp_bytes / (sms[1] / max(ssteps, 1) * 1e-3) / 1e9 / peak,
+                                          "topk_frac": tk_bytes / (sms[0] / max(ssteps, 1) * 1e-3) / 1e9 / peak}},
             "gpu_launches": launches,
             "clocks": clocks,
         }

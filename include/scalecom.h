@@ -155,6 +155,9 @@ int scalecom_reset(scalecom_ctx* ctx);
                                             chunk j = [floor(j*d/k), floor((j+1)*d/k)), and each keeps its
                                             largest-magnitude coordinate (lower index on ties).  Steps 1, 3,
                                             4, 5 are unchanged.  First use allocates 8*k bytes             */
+#define SCALECOM_OPT_KERNEL_SPANS     7  /* 1: every kernel of a step records the time from its first block's
+                                            start to its last block's end on the GPU's nanosecond timer
+                                            (two atomics per block); read with scalecom_kernel_span_ms     */
 #define SCALECOM_SELECTOR_TOPK  0
 #define SCALECOM_SELECTOR_CHUNK 1
 int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
@@ -167,8 +170,9 @@ int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */
-#define SCALECOM_Q_PHASE_STAMP0     100 /* +i, i < 10: low 32 bits of the GPU nanosecond timer when block 0 of
-                                          the last selection kernel reached phase boundary i (profiling aid)   */
+#define SCALECOM_Q_PHASE_STAMP0     100 /* +i, i < 13: low 32 bits of the GPU nanosecond timer when block 0 of
+                                          the last top-k selection kernel reached phase boundary i (profiling
+                                          aid; boundaries 0-9 in phase order, 10-12 inside the final phase)    */
 int scalecom_query(scalecom_ctx* ctx, int item, int64_t* out);
 
 /*
@@ -210,6 +214,14 @@ int scalecom_kernel_ms(scalecom_ctx* ctx, float ms[3], int32_t* nsteps);
 #define SCALECOM_STATIC_MAX_D (1 << 20)
 int scalecom_topk_static(const float* g, const float* m, int64_t d, int64_t k, int32_t* out_idx,
                          int32_t* dev_status, void* cuda_stream);
+
+/*
+ * With SCALECOM_OPT_KERNEL_SPANS on: waits for the stream and writes the in-kernel durations in
+ * milliseconds (first block start to last block end, no launch gap, no event overhead) SUMMED over the
+ * steps recorded since the previous call (at most the last 256): ms[0] selection kernel, ms[1] learner
+ * pass; *nsteps receives the number of steps summed.  BAD_STATE when the option is off.
+ */
+int scalecom_kernel_span_ms(scalecom_ctx* ctx, float ms[2], int32_t* nsteps);
 
 /* Static, never NULL. */
 const char* scalecom_strerror(int code);

@@ -21,7 +21,7 @@ ERR_INVALID_ARG, ERR_NULL_PTR, ERR_ALLOC, ERR_CUDA = -1, -2, -3, -4
 ERR_TIMEOUT, ERR_BAD_STATE, ERR_INTERNAL, ERR_ALIAS = -5, -6, -7, -8
 MAX_LEARNERS = 1024
 
-OPT_FORCE_EXACT_PATH, OPT_SPIN_LIMIT, OPT_KERNEL_TIMING, OPT_FUSE_UPDATE, OPT_USE_HINT, OPT_SELECTOR = 1, 2, 3, 4, 5, 6
+OPT_FORCE_EXACT_PATH, OPT_SPIN_LIMIT, OPT_KERNEL_TIMING, OPT_FUSE_UPDATE, OPT_USE_HINT, OPT_SELECTOR, OPT_KERNEL_SPANS = 1, 2, 3, 4, 5, 6, 7
 PATH_SAMPLED, PATH_EXACT, PATH_HINTED, PATH_CHUNK = 0, 1, 2, 3
 SELECTOR_TOPK, SELECTOR_CHUNK = 0, 1
 Q_PHASE_STAMP0 = 100
@@ -31,7 +31,7 @@ EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
     "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
-    "scalecom_topk_static",
+    "scalecom_topk_static", "scalecom_kernel_span_ms",
 )
 STATIC_MAX_D = 1 << 20
 
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.scalecom_kernel_ms.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(i32)]
         L.scalecom_topk_static.restype = ctypes.c_int
         L.scalecom_topk_static.argtypes = [vp, vp, i64, i64, vp, vp, vp]
+        L.scalecom_kernel_span_ms.restype = ctypes.c_int
+        L.scalecom_kernel_span_ms.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(i32)]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -191,6 +193,13 @@ class Context:
         ms = (ctypes.c_float * 3)()
         ns = ctypes.c_int32()
         _check(lib().scalecom_kernel_ms(self._h, ms, ctypes.byref(ns)), "scalecom_kernel_ms")
+        return list(ms), ns.value
+
+    def kernel_span_ms(self) -> Tuple[List[float], int]:
+        """(summed in-kernel milliseconds [selection, learner pass], steps summed)."""
+        ms = (ctypes.c_float * 2)()
+        ns = ctypes.c_int32()
+        _check(lib().scalecom_kernel_span_ms(self._h, ms, ctypes.byref(ns)), "scalecom_kernel_span_ms")
         return list(ms), ns.value
 
     def step(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], weights: Optional[torch.Tensor],

@@ -43,9 +43,7 @@ struct ChunkParams {
     uint32_t* ctrl;                     // status word at [CT_STATUS], path at [CT_PATH]
     unsigned long long* barrier;        // arrival counter used by this kernel only
     int32_t* out_idx;                   // [k] or nullptr
-#ifdef SC_PROFILE_SPANS
-    unsigned long long* spans;
-#endif
+    unsigned long long* spans;          // nullptr, or where to accumulate the kernel's time span
 };
 
 // Chunk of coordinate p: the j with j*d < (p+1)*k <= (j+1)*d.
@@ -67,7 +65,7 @@ __global__ void __launch_bounds__(CS_THREADS, CS_BLOCKS_PER_SM) chunk_select_ker
     const uint32_t d = P.d, k = P.k;
     GridBarrier gb;
     gb.arrive = P.barrier; gb.nblocks = nblocks; gb.status = P.ctrl + 1; gb.spin_limit = P.spin_limit;
-    SC_SPAN_BEGIN(P.spans);
+    span_begin(P.spans);
 
     // the bitmap is first written after the barrier
     {
@@ -165,7 +163,7 @@ __global__ void __launch_bounds__(CS_THREADS, CS_BLOCKS_PER_SM) chunk_select_ker
         P.tile_prefix[tile] = prefix;
     }
     if (gtid == 0) { P.ctrl[2] = 3u; P.ctrl[3] = k; }                   // path 3: chunk-wise; "candidates" = k
-    SC_SPAN_END(P.spans);
+    span_end(P.spans);
 }
 
 }  // namespace sc

@@ -68,21 +68,24 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
 
 __device__ __forceinline__ uint32_t warp_sum(uint32_t v) { return __reduce_add_sync(FULL, v); }
 
-// ---- optional in-kernel time spans (build with -DSC_PROFILE_SPANS) -----------------------------------
-// Each kernel then takes a device pointer to {earliest block start, latest block end} on the
-// nanosecond global timer, which separates kernel time from launch gaps and event overhead.
-#ifdef SC_PROFILE_SPANS
+// ---- in-kernel time spans ------------------------------------------------------------------------
+// A kernel given a non-null `sp` accumulates {~(earliest block start), latest block end} on the
+// nanosecond global timer into sp[0], sp[1] (both with atomicMax on zero-initialised words), which
+// separates kernel time from launch gaps and event overhead.  One atomic per block at each end.
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-#define SC_SPAN_BEGIN(sp) do { if ((sp) && threadIdx.x == 0) atomicMin(&(sp)[0], global_timer_ns()); } while (0)
-#define SC_SPAN_END(sp) do { if (sp) { __syncthreads(); if (threadIdx.x == 0) atomicMax(&(sp)[1], global_timer_ns()); } } while (0)
-#else
-#define SC_SPAN_BEGIN(sp) do { } while (0)
-#define SC_SPAN_END(sp) do { } while (0)
-#endif
+__device__ __forceinline__ void span_begin(unsigned long long* sp) {
+    if (sp && threadIdx.x == 0) atomicMax(&sp[0], ~global_timer_ns());
+}
+__device__ __forceinline__ void span_end(unsigned long long* sp) {
+    if (sp) {
+        __syncthreads();
+        if (threadIdx.x == 0) atomicMax(&sp[1], global_timer_ns());
+    }
+}
 
 // ---- bounded grid barrier -----------------------------------------------------------------------
 // All blocks of a cooperative launch call this the same number of times.  The

@@ -40,9 +40,7 @@ struct LearnerParams {
     int32_t* out_idx;                      // [k]: the ascending index list, written here from the ranks
     float* gathered;                       // [n * k] or nullptr
     float* weights;                        // [d] or nullptr (then Algorithm 1 line 12 is not applied here)
-#ifdef SC_PROFILE_SPANS
-    unsigned long long* spans;             // {earliest block start, latest block end}, ns
-#endif
+    unsigned long long* spans;             // nullptr, or where to accumulate the kernel's time span
 };
 
 // One burst of a thread covers LP_T consecutive tiles x LP_L learners (LP_T * LP_L = LP_UNROLL pairs of
@@ -57,9 +55,7 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
     const int n = P.n;
     const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside a tile
     const uint32_t sh = (tid & 7u) * 4u;           // and its first bit inside that word
-#ifdef SC_PROFILE_SPANS
-    SC_SPAN_BEGIN(P.spans);
-#endif
+    span_begin(P.spans);
 
     const uint32_t nsuper = (P.ntiles + LP_T - 1) / LP_T;
     for (uint32_t sup = blockIdx.x; sup < nsuper; sup += gridDim.x) {
@@ -127,9 +123,7 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                     }
             }
     }
-#ifdef SC_PROFILE_SPANS
-    SC_SPAN_END(P.spans);
-#endif
+    span_end(P.spans);
 }
 
 // Algorithm 1 line 12 as its own kernel: theta[idx[j]] -= lr * val[j].

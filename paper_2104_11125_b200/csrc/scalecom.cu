@@ -49,7 +49,10 @@ struct scalecom_ctx {
     bool timing = false;
     bool fuse_update = true;
     float* gathered = nullptr;
-    unsigned long long* spans = nullptr;     // only used by SC_PROFILE_SPANS builds
+    // in-kernel time spans: a ring of {selection ~start, end, learner pass ~start, end} per step
+    unsigned long long* spans = nullptr;     // [EV_RING * 4] device words, allocated when first switched on
+    bool span_timing = false;
+    int64_t span_steps = 0;
 
     // host-buffer entry point
     float* stage_g = nullptr;          // n*d
@@ -188,9 +191,9 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     tp.ntiles = c->ntiles;
     tp.tiles_per_block = c->tiles_per_block;
     tp.out_idx = nullptr;          // the learner pass writes the index list from the ranks it computes anyway
-#ifdef SC_PROFILE_SPANS
-    tp.spans = c->spans;
-#endif
+    unsigned long long* const span_slot =
+        (c->span_timing && c->spans) ? c->spans + 4 * (c->span_steps % scalecom_ctx::EV_RING) : nullptr;
+    tp.spans = span_slot;
 
     LearnerParams lp;
     lp.d = uint32_t(c->d);
@@ -207,9 +210,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     lp.out_idx = out_idx;
     lp.gathered = c->gathered;
     lp.weights = (weights && c->fuse_update) ? weights : nullptr;
-#ifdef SC_PROFILE_SPANS
-    lp.spans = c->spans ? c->spans + 2 : nullptr;
-#endif
+    lp.spans = span_slot ? span_slot + 2 : nullptr;
 
     bool vec_all = true;
     for (int i = 0; i < c->n; ++i) vec_all = vec_all && aligned16(grads[i]) && aligned16(mem[i]);
@@ -229,9 +230,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
         cp.ctrl = c->ctrl;
         cp.barrier = c->barrier + 8;               // its own arrival counter: the grid differs from the top-k kernel's
         cp.out_idx = nullptr;                      // written by the learner pass
-#ifdef SC_PROFILE_SPANS
-        cp.spans = c->spans;
-#endif
+        cp.spans = span_slot;
         e = vec_leader ? launch_chunk<true>(c, cp) : launch_chunk<false>(c, cp);
     } else {
         e = vec_leader ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
@@ -256,6 +255,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
         if (weights && !c->fuse_update && cudaEventRecord(ev[3], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
         ++c->ev_steps;
     }
+    if (span_slot) ++c->span_steps;
     return SCALECOM_OK;
 }
 
@@ -436,6 +436,7 @@ void scalecom_destroy(scalecom_ctx* c) {
     }
     cudaFree(c->ws);
     cudaFree(c->chunk_best);
+    cudaFree(c->spans);
     cudaFree(c->stage_g);
     cudaFree(c->stage_idx);
     cudaFree(c->stage_val);
@@ -451,11 +452,6 @@ int scalecom_set_stream(scalecom_ctx* c, void* cuda_stream) {
     return SCALECOM_OK;
 }
 
-#ifdef SC_PROFILE_SPANS
-// Profiling builds only: p points to 4 device u64 {selection start, end, learner pass start, end}
-// (initialise starts to a large value, ends to 0); nullptr switches the time spans off.
-int scalecom_profile_spans(scalecom_ctx* c, unsigned long long* p) { c->spans = p; return 0; }
-#endif
 int scalecom_set_gathered(scalecom_ctx* c, float* dev_gathered) {
     if (!c) return SCALECOM_ERR_NULL_PTR;
     c->gathered = dev_gathered;
@@ -520,6 +516,19 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
         }
         case SCALECOM_OPT_FUSE_UPDATE: c->fuse_update = value != 0; return SCALECOM_OK;
         case SCALECOM_OPT_USE_HINT: c->use_hint = value ? 1u : 0u; return SCALECOM_OK;
+        case SCALECOM_OPT_KERNEL_SPANS: {
+            DeviceGuard guard(c->device);
+            const size_t bytes = size_t(scalecom_ctx::EV_RING) * 4 * 8;
+            if (value && !c->spans && cudaMalloc(reinterpret_cast<void**>(&c->spans), bytes) != cudaSuccess) {
+                cudaGetLastError();
+                c->spans = nullptr;
+                return SCALECOM_ERR_ALLOC;
+            }
+            if (c->spans && cudaMemsetAsync(c->spans, 0, bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+            c->span_timing = value != 0;
+            c->span_steps = 0;
+            return SCALECOM_OK;
+        }
         case SCALECOM_OPT_SELECTOR: {
             if (value != SCALECOM_SELECTOR_TOPK && value != SCALECOM_SELECTOR_CHUNK) return SCALECOM_ERR_INVALID_ARG;
             if (value == SCALECOM_SELECTOR_CHUNK && !c->chunk_best) {
@@ -565,7 +574,7 @@ int scalecom_query(scalecom_ctx* c, int item, int64_t* out) {
             *out = item == SCALECOM_Q_LAST_TOPK_PATH ? w[CT_PATH] : w[CT_M];
             return SCALECOM_OK;
         default:
-            if (item >= SCALECOM_Q_PHASE_STAMP0 && item < SCALECOM_Q_PHASE_STAMP0 + 16) {
+            if (item >= SCALECOM_Q_PHASE_STAMP0 && item < SCALECOM_Q_PHASE_STAMP0 + CT_NSTAMPS) {
                 if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
                     cudaMemcpy(w, c->ctrl, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess)
                     return SCALECOM_ERR_CUDA;
@@ -594,6 +603,30 @@ int scalecom_kernel_ms(scalecom_ctx* c, float ms[3], int32_t* nsteps) {
     }
     *nsteps = int32_t(kept);
     c->ev_steps = 0;
+    return SCALECOM_OK;
+}
+
+int scalecom_kernel_span_ms(scalecom_ctx* c, float ms[2], int32_t* nsteps) {
+    if (!c || !ms || !nsteps) return SCALECOM_ERR_NULL_PTR;
+    if (!c->span_timing || !c->spans) return SCALECOM_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    static_assert(scalecom_ctx::EV_RING * 4 * 8 <= 16384, "span ring copied to the stack");
+    unsigned long long h[scalecom_ctx::EV_RING * 4];
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
+        cudaMemcpy(h, c->spans, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemset(c->spans, 0, sizeof h) != cudaSuccess)
+        return SCALECOM_ERR_CUDA;
+    const int64_t kept = c->span_steps < scalecom_ctx::EV_RING ? c->span_steps : scalecom_ctx::EV_RING;
+    double sum[2] = {0.0, 0.0};
+    for (int64_t s = 0; s < kept; ++s)
+        for (int i = 0; i < 2; ++i) {
+            const unsigned long long start = ~h[4 * s + 2 * i], end = h[4 * s + 2 * i + 1];
+            if (end > start) sum[i] += double(end - start) * 1e-6;
+        }
+    ms[0] = float(sum[0]);
+    ms[1] = float(sum[1]);
+    *nsteps = int32_t(kept);
+    c->span_steps = 0;
     return SCALECOM_OK;
 }
 

@@ -69,7 +69,7 @@ constexpr uint32_t BCAP = 1024;                                // boundary list 
 
 // ctrl words
 constexpr int CT_CAND = 0, CT_STATUS = 1, CT_PATH = 2, CT_M = 3, CT_BCOUNT = 4, CT_OVERFLOW = 5, CT_HINT = 6, CT_MARGIN = 7;
-constexpr int CT_STAMP = 8, CT_NSTAMPS = 10, CT_WORDS = 32;
+constexpr int CT_STAMP = 8, CT_NSTAMPS = 13, CT_WORDS = 32;
 // selection paths reported in ctrl[CT_PATH]
 constexpr uint32_t PATH_FAST = 0, PATH_EXACT = 1, PATH_FAST_HINT = 2;
 
@@ -98,9 +98,7 @@ struct TopkParams {
     uint32_t ntiles;
     uint32_t tiles_per_block;  // span of the final scan
     int32_t* out_idx;          // [k], or nullptr when the caller derives the index list itself
-#ifdef SC_PROFILE_SPANS
-    unsigned long long* spans;
-#endif
+    unsigned long long* spans;     // nullptr, or where to accumulate the kernel's time span
 };
 
 struct TopkShared {
@@ -238,10 +236,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                                           P.ctrl[CT_STAMP + (i)] = ts_; } } while (0)
 #define SC_BARRIER() do { if (!grid_barrier(gb, &s.flag)) return; } while (0)
 
-    SC_SPAN_BEGIN(P.spans);
-#ifdef SC_PROFILE_SPANS
-    if (P.spans && tid == 0) P.spans[4 + 2 * blockIdx.x] = global_timer_ns();     // per-block start (profiling builds)
-#endif
+    span_begin(P.spans);
     SC_STAMP(0);
     SC_STAMP(1); SC_STAMP(2); SC_STAMP(3);                             // overwritten when the sample phases run
 
@@ -714,10 +709,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
         }
     }
     SC_STAMP(9);
-#ifdef SC_PROFILE_SPANS
-    if (P.spans && tid == 0) P.spans[5 + 2 * blockIdx.x] = global_timer_ns();     // per-block end
-#endif
-    SC_SPAN_END(P.spans);
+    span_end(P.spans);
 #undef SC_BARRIER
 #undef SC_STAMP
 }

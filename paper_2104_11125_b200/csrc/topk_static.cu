@@ -152,9 +152,7 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
     }
     P.tiles_per_block = (P.ntiles + blocks - 1) / blocks;
     P.out_idx = out_idx;
-#ifdef SC_PROFILE_SPANS
     P.spans = nullptr;
-#endif
 
     // Every call shares the array and finds the previous call's contents in it: the
     // counters, the histograms and the barrier word must start at zero (the kernel

@@ -274,3 +274,28 @@ def test_switching_selectors_on_one_handle():
             idx_o, val_o, _ = oracle.step([x.cpu().numpy() for x in g], m_o, None, t, w.k, w.beta, w.lr, selector=sel)
             assert np.array_equal(idx.cpu().numpy(), idx_o) and np.array_equal(val.cpu().numpy(), val_o), (t, sel)
         assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(m, m_o))
+
+
+def test_kernel_timing_queries():
+    """Per-kernel CUDA-event times and in-kernel time spans: positive, consistent, reset on read."""
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    w = W.TINY.scaled(1_000_000)
+    prof = W.profile(w, DEV)
+    m = W.initial_memory(w, DEV)
+    idx = torch.empty(w.k, device=DEV, dtype=torch.int32)
+    val = torch.empty(w.k, device=DEV)
+    with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
+        with pytest.raises(sc.ScaleComError):
+            ctx.kernel_span_ms()                       # option off
+        ctx.set_option(binding.OPT_KERNEL_TIMING, 1)
+        ctx.set_option(binding.OPT_KERNEL_SPANS, 1)
+        for t in range(5):
+            ctx.step(W.gradients(w, t, DEV, prof), m, None, t, idx, val)
+        ev, ne = ctx.kernel_ms()
+        sp, ns = ctx.kernel_span_ms()
+        assert ne == 5 and ns == 5
+        assert 0 < sp[0] <= ev[0] * 1.05 and 0 < sp[1] <= ev[1] * 1.05     # a span lies inside its event interval
+        assert ev[2] == 0.0                                                  # weight update fused: no third kernel
+        assert ctx.kernel_ms()[1] == 0 and ctx.kernel_span_ms()[1] == 0      # both forget what they reported
+        assert ctx.status() == 0
