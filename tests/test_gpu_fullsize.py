@@ -119,3 +119,96 @@ def test_chunk_selector_full_size_every_element(w):
     from tests.parity import workload_case
     paths = workload_case(w, 2, DEV, selector="chunk")
     assert paths == [3, 3]
+
+
+def test_maximum_dimension():
+    """d = 2^31 - 1, the largest vector the ABI accepts (one learner, so 26 GB on the device).
+    The oracle cannot sort 2^31 records in a test's time, so the selection is checked through what
+    holds at any size -- the threshold property with the tie rule, counted on the device -- and
+    through the oracle's rank definition on sampled coordinates; memory, reduced values and weights
+    are compared with the oracle element by element inside windows (including the very last one)."""
+    import paper_2104_11125_b200 as sc
+    from tests.parity import rel_err, REL_TOL
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * 2 ** 30:
+        pytest.skip("needs ~50 GB of free device memory")
+    d, n, k, beta, lr = 2 ** 31 - 1, 1, (2 ** 31 - 1) // 4096, 0.25, 0.5
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(20210411)
+    g = torch.randn(d, generator=gen, device=DEV)
+    m = torch.randn(d, generator=gen, device=DEV).mul_(0.5)
+    g[-1] = 100.0                                             # the very last coordinate must be selectable
+    th = torch.zeros(d, device=DEV)
+    m0 = m.clone()
+    idx = torch.empty(k, device=DEV, dtype=torch.int32)
+    val = torch.empty(k, device=DEV)
+    with sc.Context(d, n, k, beta, lr) as ctx:
+        ctx.step([g], [m], th, 0, idx, val)
+        assert ctx.status() == 0
+    # ---- selection: properties on the device ----
+    acc = m0 + g                                              # the same fp32 sum the kernel forms
+    key = acc.view(torch.int32) & 0x7FFFFFFF
+    il = idx.long()
+    assert bool((il[1:] > il[:-1]).all()) and int(il[0]) >= 0 and int(il[-1]) == d - 1
+    sel_keys = key[il]
+    tau = int(sel_keys.min())
+    n_above = int((key > tau).sum())
+    n_at = int((key == tau).sum())
+    assert n_above < k <= n_above + n_at                      # tau is the k-th largest key
+    assert int((sel_keys > tau).sum()) == n_above             # everything above the threshold is in
+    ties = torch.nonzero(key == tau).flatten()                # among equals, the lowest indices win
+    need = k - n_above
+    assert torch.equal(torch.sort(il[sel_keys == tau]).values, ties[:need])
+    del key, sel_keys
+    # ---- selection: the oracle's rank definition on sampled coordinates ----
+    acc_h = acc.cpu().numpy()
+    del acc
+    sel = torch.zeros(d, dtype=torch.bool, device=DEV)
+    sel[il] = True
+    rng = np.random.default_rng(3)
+    picks = list(rng.integers(0, d, 3)) + [int(il[0]), int(il[k // 2]), d - 1]
+    for p in picks:
+        assert (oracle.rank(acc_h, int(p)) < k) == bool(sel[int(p)]), p
+    del acc_h
+    # ---- values, memory, weights inside windows: oracle on the slice ----
+    idx_h = idx.cpu().numpy()
+    val_h = val.cpu().numpy()
+    for a, b in [(0, WIN), (d // 2 - 7, d // 2 - 7 + WIN), (d - WIN - 1, d)]:
+        j0, j1 = np.searchsorted(idx_h, a), np.searchsorted(idx_h, b)
+        idx_w = (idx_h[j0:j1] - a).astype(np.int32)
+        sel_w = sel[a:b].cpu().numpy().astype(np.uint8)
+        m_w = m0[a:b].cpu().numpy().copy()
+        G_w = oracle.learner(g[a:b].cpu().numpy(), m_w, idx_w, sel_w, beta)
+        mg = m[a:b].cpu().numpy()
+        assert rel_err(mg, m_w) <= REL_TOL and np.array_equal(mg, m_w)
+        th_w = np.zeros(b - a, np.float32)
+        if j1 > j0:
+            val_w = oracle.reduce(np.ascontiguousarray(G_w[None, :]))
+            assert np.array_equal(val_h[j0:j1], val_w)
+            oracle.apply(th_w, idx_w, val_w, lr)
+        assert np.array_equal(th[a:b].cpu().numpy(), th_w)
+
+
+def test_maximum_dimension_chunk_selector():
+    """The chunk-wise selector at d = 2^31 - 1: its oracle is a single linear pass, so the whole
+    index list is compared."""
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2 ** 30:
+        pytest.skip("needs ~30 GB of free device memory")
+    d, k = 2 ** 31 - 1, (2 ** 31 - 1) // 1000
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(7)
+    g = torch.randn(d, generator=gen, device=DEV)
+    m = torch.zeros(d, device=DEV)
+    idx = torch.empty(k, device=DEV, dtype=torch.int32)
+    val = torch.empty(k, device=DEV)
+    acc_h = g.cpu().numpy()                                   # m = 0: acc = g exactly
+    with sc.Context(d, 1, k, 1.0, 0.0) as ctx:
+        ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK)
+        ctx.step([g], [m], None, 0, idx, val)
+        assert ctx.status() == 0
+    idx_o, _ = oracle.chunk_select(acc_h, k)
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    assert np.array_equal(val.cpu().numpy(), acc_h[idx_o])
