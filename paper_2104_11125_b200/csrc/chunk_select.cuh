@@ -20,12 +20,12 @@ namespace sc {
 #define SC_CS_THREADS 512
 #endif
 #ifndef SC_CS_BLOCKS_PER_SM
-#define SC_CS_BLOCKS_PER_SM 3
+#define SC_CS_BLOCKS_PER_SM 2
 #endif
 constexpr int CS_THREADS = SC_CS_THREADS;
 constexpr int CS_BLOCKS_PER_SM = SC_CS_BLOCKS_PER_SM;
 #ifndef SC_CS_GROUP
-#define SC_CS_GROUP 2
+#define SC_CS_GROUP 3
 #endif
 constexpr int CS_GROUP = SC_CS_GROUP;           // chunks a warp works on at a time
 constexpr int CS_UNROLL = 4;                    // rows of 32 coordinates of each of them in flight

@@ -75,6 +75,14 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
             pc[t] = have ? tile * TILE + tid * 4u : d;                 // d: nothing to do
         }
 
+        // weights at the selected coordinates, fetched now so that their latency hides behind the learner loop
+        float wv[LP_T][4];
+#pragma unroll
+        for (int t = 0; t < LP_T; ++t)
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                wv[t][c] = (P.weights && ((nib[t] >> c) & 1u) && pc[t] + c < d) ? P.weights[pc[t] + c] : 0.0f;
+
         float sum[LP_T][4];
         for (int i0 = 0; i0 < n; i0 += LP_L) {
             float gv[LP_T][LP_L][4], mv[LP_T][LP_L][4];
@@ -119,7 +127,7 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                         const float v = __fdiv_rn(sum[t][c], P.nf);                           // line 10: one division by n
                         P.out_idx[r] = int32_t(pc[t] + c);
                         P.out_val[r++] = v;
-                        if (P.weights) P.weights[pc[t] + c] = __fsub_rn(P.weights[pc[t] + c], __fmul_rn(P.lr, v));   // line 12
+                        if (P.weights) P.weights[pc[t] + c] = __fsub_rn(wv[t][c], __fmul_rn(P.lr, v));   // line 12
                     }
             }
     }
