@@ -26,7 +26,7 @@ struct scalecom_ctx {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     uint32_t *samp_hist = nullptr, *coarse_win = nullptr, *fine_hist = nullptr, *digit_hist = nullptr;
-    uint32_t *block_tot = nullptr, *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr;
+    uint32_t *block_tot = nullptr, *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr, *leader_hint = nullptr;
     unsigned long long* barrier = nullptr;
     uint2* cand = nullptr;
     uint2* blist = nullptr;
@@ -175,6 +175,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     tp.samp_target = c->samp_target;
     tp.force_exact = c->force_exact;
     tp.use_hint = c->use_hint;
+    tp.leader_hint = c->leader_hint + leader;
     tp.spin_limit = c->spin_limit;
     tp.samp_hist = c->samp_hist;
     tp.coarse_win = c->coarse_win;
@@ -339,7 +340,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     size_t off = 0;
     auto carve = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
     const size_t o_samp = carve(NCOARSE * 4), o_cw = carve((WIN + 1) * 4), o_ctrl = carve(CT_WORDS * 4), o_bar = carve(256);
-    const size_t o_bt = carve(size_t(c->topk_blocks) * 4);
+    const size_t o_bt = carve(size_t(c->topk_blocks) * 4), o_lh = carve(size_t(n) * 4);
     const size_t o_fine = carve(NFINE * 4), o_dh = carve(size_t(DH_PASSES) * DH_BINS * 4);
     c->ctrl_region_bytes = off;                 // everything the kernel expects to find zero
     const size_t o_cand = carve(size_t(c->seg_cap) * c->topk_blocks * TK_WARPS * 8), o_bl = carve(size_t(BCAP) * 8);
@@ -356,6 +357,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->ctrl = reinterpret_cast<uint32_t*>(base + o_ctrl);
     c->barrier = reinterpret_cast<unsigned long long*>(base + o_bar);
     c->block_tot = reinterpret_cast<uint32_t*>(base + o_bt);
+    c->leader_hint = reinterpret_cast<uint32_t*>(base + o_lh);
     c->fine_hist = reinterpret_cast<uint32_t*>(base + o_fine);
     c->digit_hist = reinterpret_cast<uint32_t*>(base + o_dh);
     c->cand = reinterpret_cast<uint2*>(base + o_cand);

@@ -10,8 +10,9 @@
 //   P1  every block derives from the sample a conservative lower bound on the
 //       k-th key (bin b_lo), aiming at slightly more than k survivors.
 //       P0/P1 are skipped when the previous launch of the same handle left a
-//       hint (the bin just below the one of its k-th key): consecutive steps of a
-//       training run have nearly the same threshold.  A hint that turns out useless
+//       hint (the bin just below the one of its k-th key; this leader's own from the
+//       last time it led, else the previous step's): a learner's threshold changes
+//       slowly over a training run.  A hint that turns out useless
 //       costs one wasted pass; the step then runs P0/P1 as if there had been none,
 //       and later hints of the handle keep one more bin of distance
 //   P2  stream g, m once.  A survivor (key bin >= b_lo) is appended as (key, idx)
@@ -80,7 +81,8 @@ struct TopkParams {
     uint32_t samp_stride;      // sample one granule out of this many
     uint32_t samp_target;      // wanted number of sampled keys at or above the bound
     uint32_t force_exact;
-    uint32_t use_hint;         // 1: start from the bound the previous launch left in ctrl[CT_HINT]
+    uint32_t use_hint;         // 1: start from the bound earlier launches left behind
+    uint32_t* leader_hint;     // this leader's own entry (bin + 1 of its last threshold, 0 = none), or nullptr
     uint32_t spin_limit;
     // the four histograms are all zero on entry and all zero again on exit
     uint32_t* samp_hist;       // [NCOARSE]
@@ -251,7 +253,13 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
     st.prefix = 0; st.nbits = 0; st.need = k; st.group = d;
     bool fast = false, used_hint = false;
     uint32_t b_lo = 0, M = 0;
-    const uint32_t hint = (P.force_exact || !P.use_hint) ? 0u : __ldcg(&P.ctrl[CT_HINT]);   // bin + 1, 0 = none
+    // bound to start from (bin + 1, 0 = none): what this leader's own vector gave the last time it led
+    // (learners may differ in scale), else what the previous step found
+    uint32_t hint = 0;
+    if (!P.force_exact && P.use_hint) {
+        hint = P.leader_hint ? __ldcg(P.leader_hint) : 0u;
+        if (!hint) hint = __ldcg(&P.ctrl[CT_HINT]);
+    }
 
     for (int attempt = hint ? 0 : 1; attempt < 2 && !P.force_exact; ++attempt) {
         if (attempt == 0) {
@@ -705,7 +713,9 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
             if (hint && !used_hint) P.ctrl[CT_MARGIN] = 1u;
             const uint32_t margin = 1u + ((hint && !used_hint) ? 1u : __ldcg(&P.ctrl[CT_MARGIN]));
             const uint32_t cbk = st.nbits >= 13 ? uint32_t(st.prefix >> (st.nbits - 13)) : 0u;
-            P.ctrl[CT_HINT] = cbk > margin ? cbk - margin + 1u : 0u;
+            const uint32_t next_hint = cbk > margin ? cbk - margin + 1u : 0u;
+            P.ctrl[CT_HINT] = next_hint;
+            if (P.leader_hint) *P.leader_hint = next_hint;
         }
     }
     SC_STAMP(9);

@@ -124,6 +124,7 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
     }
     P.force_exact = 0;
     P.use_hint = 0;               // the scratch is shared by unrelated callers: no carry-over between calls
+    P.leader_hint = nullptr;
     P.spin_limit = 1u << 22;
     P.samp_hist = reinterpret_cast<uint32_t*>(base + OFF_SAMP);
     P.coarse_win = reinterpret_cast<uint32_t*>(base + OFF_CW);

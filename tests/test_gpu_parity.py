@@ -220,7 +220,10 @@ def test_threshold_hint_is_used_then_survives_scale_jumps():
     scales = [1.0, 1.0, 1e-3, 1e-3, 50.0, 50.0]
     jumpy = [[g * sc for g in step] for step, sc in zip(base, scales)]
     paths = p.run_and_compare(jumpy, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.001, w.lr, tag="jumps")
-    assert paths == [0, 2, 0, 2, 0, 2], paths
+    # leaders 0,1,2,3,0,1: a step starts from its leader's own last threshold if it has one, else from the
+    # previous step's; the down-jump fails once (step 2), the up-jump once per leader that still
+    # remembers the old scale (steps 4 and 5)
+    assert paths == [0, 2, 0, 2, 0, 0], paths
 
 
 # ---- chunk-wise selector (Section 4 / Appendix E) ----------------------------------------------------
@@ -299,3 +302,17 @@ def test_kernel_timing_queries():
         assert ev[2] == 0.0                                                  # weight update fused: no third kernel
         assert ctx.kernel_ms()[1] == 0 and ctx.kernel_span_ms()[1] == 0      # both forget what they reported
         assert ctx.status() == 0
+
+
+def test_threshold_hint_with_learners_of_different_scale():
+    """Learners whose gradients differ in scale by up to 16x: a step starts from the threshold its
+    own leader had the last time it led, so from the second round of leaders on no step wastes a pass."""
+    from paper_2104_11125_b200 import binding
+    w = W.TINY.scaled(400_003)
+    prof = W.profile(w, DEV)
+    scale = [1.0, 4.0, 0.25, 2.0]
+    steps = [[g * sc for g, sc in zip(W.gradients(w, s, DEV, prof), scale)] for s in range(12)]
+    paths = _parity().run_and_compare(steps, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.001, w.lr,
+                                      tag="heterogeneous")
+    assert paths[0] == binding.PATH_SAMPLED
+    assert all(p == binding.PATH_HINTED for p in paths[w.n:]), paths
