@@ -14,7 +14,9 @@ error-feedback top-k (Remark 1), acc = sparse + residual (Eq. 4), leader
 cycling (Algorithm 1 line 6), commutativity (Eq. 1), the virtual-sequence
 identity of Appendix D.1, the contraction identity of Appendix C and a
 library top-k cross-check; the chunk-wise selector by per-chunk brute force,
-its k = d and k = 1 limits and the structure of Appendix E's demonstration.
+its k = d and k = 1 limits and the structure of Appendix E's demonstration;
+the diagnostics (all-reduced vector, Hamming distance of Eq. 5, cosine
+distance) by their closed forms and special cases.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
@@ -39,7 +41,7 @@ def build(force: bool = False) -> str:
              or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_INC)))
     if force or stale:
         tmp = _LIB + ".tmp.%d" % os.getpid()
-        subprocess.run(["gcc", *CFLAGS, _SRC, "-o", tmp], check=True, cwd=_HERE)
+        subprocess.run(["gcc", *CFLAGS, _SRC, "-o", tmp, "-lm"], check=True, cwd=_HERE)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -59,6 +61,9 @@ def _load():
             f = getattr(_lib, "oracle_chunk_select_" + sfx); f.restype = ctypes.c_int; f.argtypes = [vp, i64, i64, vp, vp]
             f = getattr(_lib, "oracle_step_sel_" + sfx); f.restype = ctypes.c_int
             f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, ctypes.c_int, vp, vp, vp]
+            f = getattr(_lib, "oracle_mean_acc_" + sfx); f.restype = None; f.argtypes = [vp, vp, i32, i64, vp]
+            f = getattr(_lib, "oracle_hamming_d_" + sfx); f.restype = i64; f.argtypes = [vp, vp, i64]
+            f = getattr(_lib, "oracle_cosine_distance_" + sfx); f.restype = ctypes.c_double; f.argtypes = [vp, vp, i64]
             f = getattr(_lib, "oracle_accumulate_" + sfx); f.restype = None; f.argtypes = [vp, vp, i64, vp]
             f = getattr(_lib, "oracle_learner_" + sfx); f.restype = None
             f.argtypes = [vp, vp, i64, vp, i64, vp, real, vp]
@@ -120,6 +125,34 @@ def chunk_select(x: np.ndarray, k: int):
     sel = np.empty(d, np.uint8)
     getattr(lib, "oracle_chunk_select_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), d, int(k), _p(idx), _p(sel))
     return idx, sel
+
+
+def mean_acc(g, m) -> np.ndarray:
+    """(1/n) sum_i (m_i + g_i), learner order, one division: the all-reduced error-feedback gradient."""
+    lib = _load()
+    n, dtype, d = len(g), g[0].dtype, g[0].size
+    for a in list(g) + list(m):
+        _chk(a, dtype, (d,))
+    gp = (ctypes.c_void_p * n)(*[_p(a) for a in g])
+    mp = (ctypes.c_void_p * n)(*[_p(a) for a in m])
+    out = np.empty(d, dtype)
+    getattr(lib, "oracle_mean_acc_" + _sfx(dtype))(ctypes.cast(gp, ctypes.c_void_p), ctypes.cast(mp, ctypes.c_void_p),
+                                                   n, d, _p(out))
+    return out
+
+
+def hamming_d(sel1: np.ndarray, sel2: np.ndarray) -> int:
+    """d of Eq. 5: half the Hamming distance between two 0/1 indicator vectors (uint8)."""
+    lib = _load()
+    _chk(sel1, np.uint8); _chk(sel2, np.uint8, sel1.shape)
+    return int(lib.oracle_hamming_d_f32(_p(sel1), _p(sel2), sel1.size))
+
+
+def cosine_distance(x: np.ndarray, y: np.ndarray) -> float:
+    """1 - x.y / (|x| |y|) (Section 2, footnote), accumulated in double."""
+    lib = _load()
+    _chk(y, x.dtype, x.shape)
+    return float(getattr(lib, "oracle_cosine_distance_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), _p(y), x.size))
 
 
 def accumulate(g: np.ndarray, m: np.ndarray) -> np.ndarray:

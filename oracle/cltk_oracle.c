@@ -8,9 +8,10 @@
  * compare the CUDA library against.  It shares no code with that library and
  * nothing in the product path may call it.
  *
- * Build:  gcc -std=c99 -O2 -ffp-contract=off -fPIC -shared cltk_oracle.c -o libcltk_oracle.so
+ * Build:  gcc -std=c99 -O2 -ffp-contract=off -fPIC -shared cltk_oracle.c -o libcltk_oracle.so -lm
  * (-ffp-contract=off: no fused multiply-add, so every operation rounds once.)
  */
+#include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>

@@ -356,3 +356,39 @@ def test_chunk_step_is_the_same_algorithm_with_another_index_set():
     x = acc[t % n]
     comp = np.zeros(d); comp[idx] = x[idx]
     np.testing.assert_allclose(np.sum((x - comp) ** 2), np.sum(x ** 2) - np.sum(x[idx] ** 2), rtol=1e-12)
+
+
+# ---- diagnostics: Eq. 5 and the cosine distance of Section 2 -------------------------------------
+def test_diagnostics_closed_forms():
+    d, k, n = 500, 40, 5
+    g = [RNG.standard_normal(d).astype(np.float32) for _ in range(n)]
+    m = [RNG.standard_normal(d).astype(np.float32) for _ in range(n)]
+    mean = oracle.mean_acc(g, m)
+    np.testing.assert_allclose(mean, np.mean([a.astype(np.float64) + b for a, b in zip(m, g)], axis=0), rtol=2e-6, atol=1e-7)
+    # the reduction of Algorithm 1 line 10 is this vector restricted to the selected coordinates
+    idx, val, _ = oracle.step(g, [a.copy() for a in m], None, 2, k, 0.5, 0.0)
+    assert np.array_equal(val, mean[idx])
+    # Eq. 5: H = 2d; identical sets d = 0, disjoint sets d = k, one swapped index d = 1
+    a = np.zeros(d, np.uint8); a[:k] = 1
+    b = np.zeros(d, np.uint8); b[k:2 * k] = 1
+    c = a.copy(); c[0] = 0; c[d - 1] = 1
+    assert oracle.hamming_d(a, a) == 0 and oracle.hamming_d(a, b) == k and oracle.hamming_d(a, c) == 1
+    _, s1 = oracle.topk(g[0], k)
+    _, s2 = oracle.topk(g[1], k)
+    i1, i2 = set(np.flatnonzero(s1)), set(np.flatnonzero(s2))
+    assert oracle.hamming_d(s1, s2) == k - len(i1 & i2) == len(i1 ^ i2) // 2
+    # with one learner the leader's set is the true top-k set
+    _, sl = oracle.topk(oracle.accumulate(g[0], m[0]), k)
+    _, st = oracle.topk(oracle.mean_acc(g[:1], m[:1]), k)
+    assert oracle.hamming_d(sl, st) == 0
+    # cosine distance: 0 for parallel, 2 for opposite, 1 for orthogonal, scale invariant
+    x = RNG.standard_normal(d)
+    y = RNG.standard_normal(d)
+    assert abs(oracle.cosine_distance(x, 3.0 * x)) < 1e-15
+    assert abs(oracle.cosine_distance(x, -0.5 * x) - 2.0) < 1e-15
+    e1 = np.zeros(d); e1[3] = 2.0
+    e2 = np.zeros(d); e2[7] = -5.0
+    assert oracle.cosine_distance(e1, e2) == 1.0
+    ref = 1.0 - float(np.dot(x, y)) / (np.linalg.norm(x) * np.linalg.norm(y))
+    assert abs(oracle.cosine_distance(x, y) - ref) < 1e-14
+    assert abs(oracle.cosine_distance(2.0 * x, 7.0 * y) - ref) < 1e-14
