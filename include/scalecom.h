@@ -216,6 +216,22 @@ int scalecom_topk_static(const float* g, const float* m, int64_t d, int64_t k, i
                          int32_t* dev_status, void* cuda_stream);
 
 /*
+ * Diagnostics of Sections 2-3; they read the state and change none of it (scratch of about 8.2*d
+ * bytes is allocated on first use; both calls wait for the stream).
+ *
+ * scalecom_overlap: Eq. 5's d between the leader's top-k set I^k(acc_L), L = t mod n, and the "true
+ * top-k" set I^k((1/n) sum_i acc_i) of the all-reduced error-feedback gradient: the Hamming distance of
+ * the two indicator vectors is H = 2d, 0 <= d <= k (Fig. 3 plots d/k; Lemma 1 turns it into the
+ * contraction factor).  grads / mem as in scalecom_step, all read only.
+ *
+ * scalecom_cosine_distance: 1 - x.y / (|x| |y|) of two DEVICE fp32[d] vectors, e.g. two learners'
+ * memories (Section 2, "memory similarity"); products accumulated in double.
+ */
+int scalecom_overlap(scalecom_ctx* ctx, const float* const* grads, const float* const* mem, int64_t t,
+                     int64_t* host_hamming_d);
+int scalecom_cosine_distance(scalecom_ctx* ctx, const float* x, const float* y, double* host_out);
+
+/*
  * With SCALECOM_OPT_KERNEL_SPANS on: waits for the stream and writes the in-kernel durations in
  * milliseconds (first block start to last block end, no launch gap, no event overhead) SUMMED over the
  * steps recorded since the previous call (at most the last 256): ms[0] selection kernel, ms[1] learner

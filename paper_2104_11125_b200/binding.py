@@ -31,7 +31,7 @@ EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
     "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
-    "scalecom_topk_static", "scalecom_kernel_span_ms",
+    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance",
 )
 STATIC_MAX_D = 1 << 20
 
@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.scalecom_topk_static.argtypes = [vp, vp, i64, i64, vp, vp, vp]
         L.scalecom_kernel_span_ms.restype = ctypes.c_int
         L.scalecom_kernel_span_ms.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(i32)]
+        L.scalecom_overlap.restype = ctypes.c_int
+        L.scalecom_overlap.argtypes = [vp, vp, vp, i64, ctypes.POINTER(i64)]
+        L.scalecom_cosine_distance.restype = ctypes.c_int
+        L.scalecom_cosine_distance.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_double)]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -201,6 +205,21 @@ class Context:
         ns = ctypes.c_int32()
         _check(lib().scalecom_kernel_span_ms(self._h, ms, ctypes.byref(ns)), "scalecom_kernel_span_ms")
         return list(ms), ns.value
+
+    def overlap(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], t: int) -> int:
+        """Eq. 5's d between the leader's top-k set and the true top-k set (synchronous)."""
+        gp = _ptr_array([_dev_f32(g, self.d, "grads[%d]" % i) for i, g in enumerate(grads)])
+        mp = _ptr_array([_dev_f32(m, self.d, "mem[%d]" % i) for i, m in enumerate(mem)])
+        out = ctypes.c_int64()
+        _check(lib().scalecom_overlap(self._h, ctypes.cast(gp, ctypes.c_void_p), ctypes.cast(mp, ctypes.c_void_p),
+                                      int(t), ctypes.byref(out)), "scalecom_overlap")
+        return out.value
+
+    def cosine_distance(self, x: torch.Tensor, y: torch.Tensor) -> float:
+        out = ctypes.c_double()
+        _check(lib().scalecom_cosine_distance(self._h, _dev_f32(x, self.d, "x"), _dev_f32(y, self.d, "y"),
+                                              ctypes.byref(out)), "scalecom_cosine_distance")
+        return out.value
 
     def step(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], weights: Optional[torch.Tensor],
              t: int, out_idx: torch.Tensor, out_val: torch.Tensor) -> None:

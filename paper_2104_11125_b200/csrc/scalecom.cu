@@ -10,6 +10,7 @@
 #include <new>
 
 #include "chunk_select.cuh"
+#include "diagnostics.cuh"
 #include "learner_pass.cuh"
 #include "topk_select.cuh"
 
@@ -66,6 +67,12 @@ struct scalecom_ctx {
     bool ev_has_update[EV_RING] = {};  // whether the step recorded the fourth event
     bool poisoned = false;
     int64_t launches = 0;
+
+    // diagnostics scratch, allocated on first use
+    float* diag_mean = nullptr;        // [d]
+    float* diag_zero = nullptr;        // [d], all zero
+    uint32_t* diag_bitmap = nullptr;   // [ntiles * 32]
+    double* diag_acc = nullptr;        // [4]: overlap count (as u64) and three dot products
 };
 
 namespace {
@@ -162,20 +169,18 @@ int check_step_args(scalecom_ctx* c, const void* const* grads, const void* const
     return SCALECOM_OK;
 }
 
-int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float* weights, int64_t t, int32_t* out_idx,
-            float* out_val) {
-    const int leader = int(t % c->n);
-
+TopkParams make_topk_params(const scalecom_ctx* c, const float* g, const float* m, uint32_t* leader_hint, bool use_hint,
+                            unsigned long long* span_slot) {
     TopkParams tp;
-    tp.g = grads[leader];
-    tp.m = mem[leader];
+    tp.g = g;
+    tp.m = m;
     tp.d = uint32_t(c->d);
     tp.k = uint32_t(c->k);
     tp.samp_stride = c->samp_stride;
     tp.samp_target = c->samp_target;
     tp.force_exact = c->force_exact;
-    tp.use_hint = c->use_hint;
-    tp.leader_hint = c->leader_hint + leader;
+    tp.use_hint = use_hint ? c->use_hint : 0u;
+    tp.leader_hint = leader_hint;
     tp.spin_limit = c->spin_limit;
     tp.samp_hist = c->samp_hist;
     tp.coarse_win = c->coarse_win;
@@ -192,9 +197,17 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     tp.ntiles = c->ntiles;
     tp.tiles_per_block = c->tiles_per_block;
     tp.out_idx = nullptr;          // the learner pass writes the index list from the ranks it computes anyway
+    tp.spans = span_slot;
+    return tp;
+}
+
+int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float* weights, int64_t t, int32_t* out_idx,
+            float* out_val) {
+    const int leader = int(t % c->n);
+
     unsigned long long* const span_slot =
         (c->span_timing && c->spans) ? c->spans + 4 * (c->span_steps % scalecom_ctx::EV_RING) : nullptr;
-    tp.spans = span_slot;
+    const TopkParams tp = make_topk_params(c, grads[leader], mem[leader], c->leader_hint + leader, true, span_slot);
 
     LearnerParams lp;
     lp.d = uint32_t(c->d);
@@ -439,6 +452,10 @@ void scalecom_destroy(scalecom_ctx* c) {
     cudaFree(c->ws);
     cudaFree(c->chunk_best);
     cudaFree(c->spans);
+    cudaFree(c->diag_mean);
+    cudaFree(c->diag_zero);
+    cudaFree(c->diag_bitmap);
+    cudaFree(c->diag_acc);
     cudaFree(c->stage_g);
     cudaFree(c->stage_idx);
     cudaFree(c->stage_val);
@@ -605,6 +622,109 @@ int scalecom_kernel_ms(scalecom_ctx* c, float ms[3], int32_t* nsteps) {
     }
     *nsteps = int32_t(kept);
     c->ev_steps = 0;
+    return SCALECOM_OK;
+}
+
+extern "C++" {
+namespace {
+
+int ensure_diag(scalecom_ctx* c) {
+    if (c->diag_mean) return SCALECOM_OK;
+    const size_t vec = size_t(c->d) * 4, bm = size_t(c->ntiles) * 32 * 4;
+    if (cudaMalloc(reinterpret_cast<void**>(&c->diag_mean), vec) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&c->diag_zero), vec) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&c->diag_bitmap), bm) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&c->diag_acc), 4 * sizeof(double)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(c->diag_mean); cudaFree(c->diag_zero); cudaFree(c->diag_bitmap); cudaFree(c->diag_acc);
+        c->diag_mean = c->diag_zero = nullptr; c->diag_bitmap = nullptr; c->diag_acc = nullptr;
+        return SCALECOM_ERR_ALLOC;
+    }
+    if (cudaMemsetAsync(c->diag_zero, 0, vec, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    return SCALECOM_OK;
+}
+
+template <int N, bool VEC>
+cudaError_t launch_mean(const scalecom_ctx* c, const float* const* grads, const float* const* mem) {
+    PtrTable<N> tab;
+    for (int i = 0; i < N; ++i) {
+        tab.g[i] = i < c->n ? grads[i] : nullptr;
+        tab.m[i] = i < c->n ? const_cast<float*>(mem[i]) : nullptr;
+    }
+    const uint32_t quads = uint32_t((c->d + 3) / 4);
+    const uint32_t want = (quads + 255u) / 256u, cap = uint32_t(c->sms) * 8u;
+    mean_acc_kernel<N, VEC><<<want < cap ? want : cap, 256, 0, c->stream>>>(tab, c->n, uint32_t(c->d), float(c->n), c->diag_mean);
+    return cudaGetLastError();
+}
+
+template <bool VEC>
+cudaError_t launch_mean_n(const scalecom_ctx* c, const float* const* grads, const float* const* mem) {
+    if (c->n <= 16) return launch_mean<16, VEC>(c, grads, mem);
+    if (c->n <= 128) return launch_mean<128, VEC>(c, grads, mem);
+    return launch_mean<SCALECOM_MAX_LEARNERS, VEC>(c, grads, mem);
+}
+
+}  // namespace
+}  // extern "C++"
+
+int scalecom_overlap(scalecom_ctx* c, const float* const* grads, const float* const* mem, int64_t t, int64_t* host_hamming_d) {
+    if (!c || !grads || !mem || !host_hamming_d) return SCALECOM_ERR_NULL_PTR;
+    if (t < 0) return SCALECOM_ERR_INVALID_ARG;
+    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
+    for (int i = 0; i < c->n; ++i)
+        if (!grads[i] || !mem[i]) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    int rc = ensure_diag(c);
+    if (rc != SCALECOM_OK) return rc;
+    const int leader = int(t % c->n);
+    const size_t bm_words = size_t(c->ntiles) * 32;
+    bool vec_all = true;
+    for (int i = 0; i < c->n; ++i) vec_all = vec_all && aligned16(grads[i]) && aligned16(mem[i]);
+
+    // leader's set I^k(acc_L): the exact selector, hints neither used nor left behind
+    TopkParams tp = make_topk_params(c, grads[leader], mem[leader], nullptr, false, nullptr);
+    cudaError_t e = (aligned16(tp.g) && aligned16(tp.m)) ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
+    if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (cudaMemcpyAsync(c->diag_bitmap, c->bitmap, bm_words * 4, cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
+        return SCALECOM_ERR_CUDA;
+    // true top-k: the same selection on the all-reduced vector
+    e = vec_all ? launch_mean_n<true>(c, grads, mem) : launch_mean_n<false>(c, grads, mem);
+    if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
+    tp = make_topk_params(c, c->diag_mean, c->diag_zero, nullptr, false, nullptr);
+    if (launch_topk<true>(c, tp) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    if (cudaMemsetAsync(c->diag_acc, 0, 4 * sizeof(double), c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    const uint32_t want = uint32_t((bm_words + 255) / 256), cap = uint32_t(c->sms) * 8u;
+    overlap_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(c->diag_bitmap, c->bitmap, bm_words,
+                                                                  reinterpret_cast<unsigned long long*>(c->diag_acc));
+    if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+    c->launches += 4;
+    unsigned long long common = 0;
+    if (cudaMemcpyAsync(&common, c->diag_acc, 8, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+        return SCALECOM_ERR_CUDA;
+    rc = scalecom_status(c);
+    if (rc != SCALECOM_OK) return rc;
+    *host_hamming_d = c->k - int64_t(common);
+    return SCALECOM_OK;
+}
+
+int scalecom_cosine_distance(scalecom_ctx* c, const float* x, const float* y, double* host_out) {
+    if (!c || !x || !y || !host_out) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    const int rc = ensure_diag(c);
+    if (rc != SCALECOM_OK) return rc;
+    if (cudaMemsetAsync(c->diag_acc, 0, 4 * sizeof(double), c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    const uint32_t want = uint32_t((c->d + 255) / 256), cap = uint32_t(c->sms) * 8u;
+    dot3_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(x, y, uint32_t(c->d), c->diag_acc + 1);
+    if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+    ++c->launches;
+    double h[3];
+    if (cudaMemcpyAsync(h, c->diag_acc + 1, sizeof h, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+        return SCALECOM_ERR_CUDA;
+    *host_out = 1.0 - h[0] / (std::sqrt(h[1]) * std::sqrt(h[2]));
     return SCALECOM_OK;
 }
 

@@ -709,6 +709,8 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
         if (pass) zero_words(P.digit_hist, size_t(pass) * DH_BINS, gtid, gsize);
         if (gtid == 0) {
             P.ctrl[CT_CAND] = 0; P.ctrl[CT_OVERFLOW] = 0;
+        }
+        if (gtid == 0 && P.use_hint) {
             // one 13-bit bin (4.4 % in magnitude) below the bin of the k-th key just found; two once a hint failed
             if (hint && !used_hint) P.ctrl[CT_MARGIN] = 1u;
             const uint32_t margin = 1u + ((hint && !used_hint) ? 1u : __ldcg(&P.ctrl[CT_MARGIN]));

@@ -316,3 +316,40 @@ def test_threshold_hint_with_learners_of_different_scale():
                                       tag="heterogeneous")
     assert paths[0] == binding.PATH_SAMPLED
     assert all(p == binding.PATH_HINTED for p in paths[w.n:]), paths
+
+
+# ---- diagnostics: Eq. 5 and the cosine distance -----------------------------------------------------
+@pytest.mark.parametrize("base,d,n", [(W.TINY, 500_003, 4), (W.RESNET50, 1_000_001, 8), (W.TRANSFORMER, 300_000, 16)])
+def test_diagnostics_match_oracle(base, d, n):
+    import paper_2104_11125_b200 as sc
+    import oracle
+    w = base.scaled(d, n=n)
+    prof = W.profile(w, DEV)
+    m = W.initial_memory(w, DEV)
+    m_o = [x.cpu().numpy().copy() for x in m]
+    idx = torch.empty(w.k, device=DEV, dtype=torch.int32)
+    val = torch.empty(w.k, device=DEV)
+    with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
+        for t in range(3):
+            g = W.gradients(w, t, DEV, prof)
+            g_np = [x.cpu().numpy() for x in g]
+            before = [x.clone() for x in m]
+            # Eq. 5 between the leader's set and the true top-k set, on the state before the step
+            L = t % w.n
+            _, sel_leader = oracle.topk(oracle.accumulate(g_np[L], m_o[L]), w.k)
+            _, sel_true = oracle.topk(oracle.mean_acc(g_np, m_o), w.k)
+            assert ctx.overlap(g, m, t) == oracle.hamming_d(sel_leader, sel_true)
+            assert all(torch.equal(a, b) for a, b in zip(m, before))          # a diagnostic changes nothing
+            if t:
+                got = ctx.cosine_distance(m[0], m[1])
+                want = oracle.cosine_distance(m_o[0], m_o[1])
+                assert abs(got - want) <= 1e-10 * max(1.0, abs(want))
+            ctx.step(g, m, None, t, idx, val)
+            idx_o, val_o, _ = oracle.step(g_np, m_o, None, t, w.k, w.beta, w.lr)
+            assert np.array_equal(idx.cpu().numpy(), idx_o) and np.array_equal(val.cpu().numpy(), val_o)
+        assert ctx.status() == 0
+    # one learner: the leader's set is the true top-k set
+    w1 = base.scaled(100_000, n=1)
+    g = W.gradients(w1, 0, DEV)
+    with sc.Context(w1.d, 1, w1.k, 0.5, 0.1) as ctx:
+        assert ctx.overlap(g, W.initial_memory(w1, DEV), 0) == 0
