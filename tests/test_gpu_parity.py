@@ -353,3 +353,33 @@ def test_diagnostics_match_oracle(base, d, n):
     g = W.gradients(w1, 0, DEV)
     with sc.Context(w1.d, 1, w1.k, 0.5, 0.1) as ctx:
         assert ctx.overlap(g, W.initial_memory(w1, DEV), 0) == 0
+
+
+@pytest.mark.parametrize("force_exact", [False, True])
+def test_non_finite_inputs_follow_the_key_order(force_exact):
+    """Keys are the bit patterns of |acc|, so +-Inf rank above every finite value and NaN above Inf,
+    deterministically; the rest of the step is plain IEEE arithmetic on both sides."""
+    import paper_2104_11125_b200 as sc
+    import oracle
+    from paper_2104_11125_b200 import binding
+    rng = np.random.default_rng(21)
+    d, n, k = 40_000, 3, 400
+    g = [rng.standard_normal(d).astype(np.float32) for _ in range(n)]
+    g[0][[5, 17_000, 39_999]] = [np.inf, -np.inf, np.nan]        # learner 0 leads at t = 0
+    g[1][123] = np.inf                                            # a non-leader's infinity is just a value
+    m = [np.zeros(d, np.float32) for _ in range(n)]
+    th = np.zeros(d, np.float32)
+    gd, md, thd = [_t(x) for x in g], [_t(x) for x in m], _t(th)
+    idx = torch.empty(k, device=DEV, dtype=torch.int32)
+    val = torch.empty(k, device=DEV)
+    with sc.Context(d, n, k, 0.5, 0.25) as ctx:
+        ctx.set_option(binding.OPT_FORCE_EXACT_PATH, int(force_exact))
+        ctx.step(gd, md, thd, 0, idx, val)
+        assert ctx.status() == 0
+    idx_o, val_o, _ = oracle.step(g, m, th, 0, k, 0.5, 0.25)
+    assert {5, 17_000, 39_999} <= set(idx_o.tolist())
+    assert np.array_equal(idx.cpu().numpy(), idx_o)
+    assert np.array_equal(val.cpu().numpy(), val_o, equal_nan=True)
+    for a, b in zip(md, m):
+        assert np.array_equal(a.cpu().numpy(), b, equal_nan=True)
+    assert np.array_equal(thd.cpu().numpy(), th, equal_nan=True)
