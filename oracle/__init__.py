@@ -61,6 +61,10 @@ def _load():
             f = getattr(_lib, "oracle_chunk_select_" + sfx); f.restype = ctypes.c_int; f.argtypes = [vp, i64, i64, vp, vp]
             f = getattr(_lib, "oracle_step_sel_" + sfx); f.restype = ctypes.c_int
             f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, ctypes.c_int, vp, vp, vp]
+            f = getattr(_lib, "oracle_layer_chunk_select_" + sfx); f.restype = ctypes.c_int
+            f.argtypes = [vp, i32, vp, vp, vp, vp]
+            f = getattr(_lib, "oracle_step_layers_" + sfx); f.restype = ctypes.c_int
+            f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, ctypes.c_int, i32, vp, vp, vp, vp, vp]
             f = getattr(_lib, "oracle_mean_acc_" + sfx); f.restype = None; f.argtypes = [vp, vp, i32, i64, vp]
             f = getattr(_lib, "oracle_hamming_d_" + sfx); f.restype = i64; f.argtypes = [vp, vp, i64]
             f = getattr(_lib, "oracle_cosine_distance_" + sfx); f.restype = ctypes.c_double; f.argtypes = [vp, vp, i64]
@@ -127,6 +131,19 @@ def chunk_select(x: np.ndarray, k: int):
     return idx, sel
 
 
+def layer_chunk_select(x: np.ndarray, sizes, keep):
+    """Chunk-wise selection with per-layer rates (Section 4): layer s has sizes[s] coordinates and
+    keeps keep[s]; returns (idx int32[sum keep] ascending, sel uint8[d])."""
+    lib = _load()
+    sz = np.ascontiguousarray(sizes, np.int64)
+    kp = np.ascontiguousarray(keep, np.int64)
+    assert sz.sum() == x.size and sz.size == kp.size and np.all(kp >= 1) and np.all(kp <= sz)
+    idx = np.empty(int(kp.sum()), np.int32)
+    sel = np.empty(x.size, np.uint8)
+    getattr(lib, "oracle_layer_chunk_select_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), sz.size, _p(sz), _p(kp), _p(idx), _p(sel))
+    return idx, sel
+
+
 def mean_acc(g, m) -> np.ndarray:
     """(1/n) sum_i (m_i + g_i), learner order, one division: the all-reduced error-feedback gradient."""
     lib = _load()
@@ -190,8 +207,9 @@ def apply(theta: np.ndarray, idx: np.ndarray, val: np.ndarray, lr: float) -> Non
 
 
 def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: bool = True,
-         selector: str = "topk"):
-    """One iteration of Algorithm 1 ("topk": Eq. 2 on the leader; "chunk": chunk-wise selection).
+         selector: str = "topk", layers=None):
+    """One iteration of Algorithm 1 ("topk": Eq. 2 on the leader; "chunk": chunk-wise selection,
+    with per-layer rates when layers = (sizes, keep) is given).
 
     g, m: lists of n ndarrays of d values (m updated in place); theta: ndarray
     of d values updated in place, or None.  Returns (idx, val, G) with G the
@@ -210,10 +228,17 @@ def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: boo
     idx = np.empty(k, np.int32)
     val = np.empty(k, dtype)
     G = np.empty((n, k), dtype) if want_gathered else None
-    rc = getattr(lib, "oracle_step_sel_" + _sfx(dtype))(
+    if layers is not None:
+        sz = np.ascontiguousarray(layers[0], np.int64)
+        kp = np.ascontiguousarray(layers[1], np.int64)
+        assert selector == "chunk" and sz.sum() == d and kp.sum() == k and sz.size == kp.size
+        nl, szp, kpp = sz.size, _p(sz), _p(kp)
+    else:
+        nl, szp, kpp = 0, None, None
+    rc = getattr(lib, "oracle_step_layers_" + _sfx(dtype))(
         ctypes.cast(gp, ctypes.c_void_p), ctypes.cast(mp, ctypes.c_void_p),
         _p(theta) if theta is not None else None,
-        int(t), n, d, int(k), float(beta), float(lr), SELECTORS[selector], _p(idx), _p(val),
+        int(t), n, d, int(k), float(beta), float(lr), SELECTORS[selector], nl, szp, kpp, _p(idx), _p(val),
         _p(G) if G is not None else None)
     if rc != 0:
         raise MemoryError("oracle_step")

@@ -392,3 +392,32 @@ def test_diagnostics_closed_forms():
     ref = 1.0 - float(np.dot(x, y)) / (np.linalg.norm(x) * np.linalg.norm(y))
     assert abs(oracle.cosine_distance(x, y) - ref) < 1e-14
     assert abs(oracle.cosine_distance(2.0 * x, 7.0 * y) - ref) < 1e-14
+
+
+# ---- chunk-wise selection with per-layer rates (Section 4) ---------------------------------------
+def test_layer_chunk_select():
+    sizes = [7, 64, 1, 300, 128]
+    keep = [7, 2, 1, 3, 16]                    # uncompressed layer, 32X, a single coordinate, 100X, 8X
+    d = sum(sizes)
+    x = RNG.standard_normal(d).astype(np.float32)
+    x[80:90] = 0.0                              # a run of ties inside a layer
+    idx, sel = oracle.layer_chunk_select(x, sizes, keep)
+    assert idx.size == sum(keep) and np.all(np.diff(idx) > 0) and sel.sum() == sum(keep)
+    key = key32(x).astype(np.int64)
+    off, expect = 0, []
+    for sz, kp in zip(sizes, keep):             # brute force: per layer, per chunk, largest magnitude then lowest index
+        for j in range(kp):
+            lo, hi = off + (j * sz) // kp, off + ((j + 1) * sz) // kp
+            expect.append(max(range(lo, hi), key=lambda p: (key[p], -p)))
+        off += sz
+    assert idx.tolist() == expect
+    assert idx[:7].tolist() == list(range(7))                          # keep = size: the layer is sent whole
+    # one layer is the plain chunk-wise selector
+    assert np.array_equal(oracle.layer_chunk_select(x, [d], [13])[0], oracle.chunk_select(x, 13)[0])
+    # the step with layers is the same algorithm with that index set
+    g = [RNG.standard_normal(d) for _ in range(3)]
+    m = [RNG.standard_normal(d) for _ in range(3)]
+    acc = np.stack([a + b for a, b in zip(m, g)])
+    idx2, val, G = oracle.step(g, [a.copy() for a in m], None, 4, sum(keep), 0.5, 0.0, selector="chunk", layers=(sizes, keep))
+    assert np.array_equal(idx2, oracle.layer_chunk_select(acc[4 % 3].copy(), sizes, keep)[0])
+    np.testing.assert_allclose(val, acc[:, idx2].mean(axis=0), rtol=1e-13)
