@@ -45,6 +45,9 @@ def parse_args():
                          "the footprint low for profiler captures")
     ap.add_argument("--selector", default="topk", choices=["topk", "chunk"],
                     help="leader selection: exact top-k (the headline path) or the chunk-wise selector")
+    ap.add_argument("--layers", action="store_true",
+                    help="with --selector chunk on a ResNet-50-shaped workload: the paper's per-layer rate rule "
+                         "(25X / 50X / 400X, first layer whole) instead of one rate; k becomes the sum of the layers' keeps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -180,7 +183,7 @@ def run_reference(args):
     }))
 
 
-def time_oracle(w, batches_dev, steps=2, selector="topk"):
+def time_oracle(w, batches_dev, steps=2, selector="topk", layers=None):
     """cpu_baseline leg: the oracle on full-size steps of the bench workload, on this machine's host cores."""
     import numpy as np
     import oracle
@@ -190,7 +193,7 @@ def time_oracle(w, batches_dev, steps=2, selector="topk"):
     for s in range(steps):
         g = [x.cpu().numpy() for x in batches_dev[s % len(batches_dev)]]
         t0 = time.perf_counter()
-        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False, selector=selector)
+        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False, selector=selector, layers=layers)
         dt += time.perf_counter() - t0
     return {"value": w.n * w.d * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
             "sample": "%d full steps of the bench workload (n=%d, d=%d, k=%d), %.1f s" % (steps, w.n, w.d, w.k, dt)}
@@ -223,6 +226,12 @@ def main():
         torch.cuda.synchronize()
 
     w = get_workload(args.workload)
+    layers = None
+    if args.layers:
+        if args.selector != "chunk" or w.kind != "resnet50":
+            raise SystemExit("--layers needs --selector chunk and a ResNet-50-shaped workload")
+        layers = W.resnet50_layer_keep(w)
+        w = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(layers[1]), w.beta, w.lr, w.steps, w.c)
     K, Wm = args.steps, max(args.warmup, 3)
     prof = W.profile(w, dev)
     nb = max(1, min(K + Wm, args.batches, MAX_BATCHES))
@@ -236,6 +245,8 @@ def main():
     ctx = sc.Context(w.d, w.n, w.k, w.beta, w.lr, stream=stream)
     if args.selector == "chunk":
         ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK)
+    if layers is not None:
+        ctx.set_layers(*layers)
     torch.cuda.synchronize()
 
     # ---- device-resident timing ---------------------------------------------------------------------
@@ -346,7 +357,7 @@ def main():
                           "h2d_bytes_per_step": 4 * w.n * w.d, "d2h_bytes_per_step": 8 * w.k,
                           "ms_per_step": e2e_ms, "api": "scalecom_step_host (pinned host gradients in, idx/val out)"}
         if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = time_oracle(w, batches, selector=args.selector)
+            out["cpu_baseline"] = time_oracle(w, batches, selector=args.selector, layers=layers)
         print(json.dumps(out))
     ctx.close()
     if world > 1:

@@ -122,6 +122,18 @@ int scalecom_set_stream(scalecom_ctx* ctx, void* cuda_stream);
 int scalecom_set_gathered(scalecom_ctx* ctx, float* dev_gathered);
 
 /*
+ * Per-layer compression rates for the chunk-wise selector (Section 4: the rate of a layer follows its
+ * FLOPs per gradient -- 25X, 50X or 400X -- and the first layer is sent uncompressed).  The d
+ * coordinates are the concatenation of nlayers layers; layer s has sizes[s] coordinates and keeps
+ * keep[s] of them by the chunk-wise rule applied inside the layer (keep[s] == sizes[s]: sent whole).
+ *   nlayers  1 .. 2048, or 0 to go back to one rate for the whole vector.
+ *   sizes, keep  HOST int64[nlayers]; sizes[s] >= 1, 1 <= keep[s] <= sizes[s], sum sizes = d, sum keep = k.
+ * Only SCALECOM_SELECTOR_CHUNK looks at the layers; the exact top-k selector ignores them.
+ * Waits for the stream.  Errors: NULL_PTR, INVALID_ARG, ALLOC, CUDA.
+ */
+int scalecom_set_layers(scalecom_ctx* ctx, int32_t nlayers, const int64_t* sizes, const int64_t* keep);
+
+/*
  * Algorithm 1 line 12 on its own: theta[idx[j]] <- theta[idx[j]] - lr * val[j]
  * for j < k, on the handle's stream, for callers that ran scalecom_step with
  * weights == NULL.  All pointers DEVICE; idx entries must be distinct and < d.

@@ -31,7 +31,7 @@ EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
     "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
-    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance",
+    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance", "scalecom_set_layers",
 )
 STATIC_MAX_D = 1 << 20
 
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.scalecom_overlap.argtypes = [vp, vp, vp, i64, ctypes.POINTER(i64)]
         L.scalecom_cosine_distance.restype = ctypes.c_int
         L.scalecom_cosine_distance.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_double)]
+        L.scalecom_set_layers.restype = ctypes.c_int
+        L.scalecom_set_layers.argtypes = [vp, i32, vp, vp]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -205,6 +207,18 @@ class Context:
         ns = ctypes.c_int32()
         _check(lib().scalecom_kernel_span_ms(self._h, ms, ctypes.byref(ns)), "scalecom_kernel_span_ms")
         return list(ms), ns.value
+
+    def set_layers(self, sizes: Optional[Sequence[int]], keep: Optional[Sequence[int]] = None) -> None:
+        """Per-layer rates of the chunk-wise selector; None goes back to one rate for the whole vector."""
+        if sizes is None:
+            _check(lib().scalecom_set_layers(self._h, 0, None, None), "scalecom_set_layers")
+            return
+        if keep is None or len(keep) != len(sizes):
+            raise ValueError("sizes and keep must have the same length")
+        sz = (ctypes.c_int64 * len(sizes))(*[int(x) for x in sizes])
+        kp = (ctypes.c_int64 * len(keep))(*[int(x) for x in keep])
+        _check(lib().scalecom_set_layers(self._h, len(sizes), ctypes.cast(sz, ctypes.c_void_p),
+                                         ctypes.cast(kp, ctypes.c_void_p)), "scalecom_set_layers")
 
     def overlap(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], t: int) -> int:
         """Eq. 5's d between the leader's top-k set and the true top-k set (synchronous)."""

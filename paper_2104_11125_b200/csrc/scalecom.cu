@@ -46,6 +46,9 @@ struct scalecom_ctx {
     int selector = SCALECOM_SELECTOR_TOPK;
     unsigned long long* chunk_best = nullptr;   // [k], allocated when the chunk-wise selector is first chosen
     uint32_t chunk_blocks = 0;
+    uint32_t nlayers = 0;              // per-layer rates of the chunk-wise selector (0: one rate for the whole vector)
+    uint32_t* layer_tab = nullptr;     // device [2][nlayers + 1]: coordinate offsets, chunk offsets
+    uint32_t* one_layer_tab = nullptr; // device {0, d, 0, k}: the whole vector as one layer
     uint32_t spin_limit = 1u << 22;
     bool timing = false;
     bool fuse_update = true;
@@ -103,8 +106,9 @@ cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
 template <bool VEC>
 cudaError_t launch_chunk(const scalecom_ctx* c, const ChunkParams& P) {
     void* args[] = {const_cast<ChunkParams*>(&P)};
-    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&chunk_select_kernel<VEC>), dim3(c->chunk_blocks),
-                                       dim3(CS_THREADS), args, 0, c->stream);
+    const void* fn = P.nl > 1 ? reinterpret_cast<const void*>(&chunk_select_kernel<VEC, true>)
+                              : reinterpret_cast<const void*>(&chunk_select_kernel<VEC, false>);
+    return cudaLaunchCooperativeKernel(fn, dim3(c->chunk_blocks), dim3(CS_THREADS), args, 0, c->stream);
 }
 
 template <int N, bool VEC, int T>
@@ -237,7 +241,6 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     if (c->selector == SCALECOM_SELECTOR_CHUNK) {
         ChunkParams cp;
         cp.g = tp.g; cp.m = tp.m; cp.d = tp.d; cp.k = tp.k;
-        cp.inv_d = 1.0 / double(c->d);
         cp.spin_limit = c->spin_limit;
         cp.best = c->chunk_best;
         cp.bitmap = c->bitmap; cp.tile_prefix = c->tile_prefix; cp.ntiles = c->ntiles;
@@ -245,6 +248,10 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
         cp.barrier = c->barrier + 8;               // its own arrival counter: the grid differs from the top-k kernel's
         cp.out_idx = nullptr;                      // written by the learner pass
         cp.spans = span_slot;
+        // one layer spanning the whole vector unless the caller set per-layer rates
+        cp.nl = c->nlayers ? c->nlayers : 1u;
+        cp.layer_off = c->nlayers ? c->layer_tab : c->one_layer_tab;
+        cp.layer_chunk0 = cp.layer_off + (cp.nl + 1);
         e = vec_leader ? launch_chunk<true>(c, cp) : launch_chunk<false>(c, cp);
     } else {
         e = vec_leader ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
@@ -451,6 +458,8 @@ void scalecom_destroy(scalecom_ctx* c) {
     }
     cudaFree(c->ws);
     cudaFree(c->chunk_best);
+    cudaFree(c->layer_tab);
+    cudaFree(c->one_layer_tab);
     cudaFree(c->spans);
     cudaFree(c->diag_mean);
     cudaFree(c->diag_zero);
@@ -469,6 +478,53 @@ int scalecom_set_stream(scalecom_ctx* c, void* cuda_stream) {
     if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;   // scratch is shared between steps
     c->stream = static_cast<cudaStream_t>(cuda_stream);
     return SCALECOM_OK;
+}
+
+int scalecom_set_layers(scalecom_ctx* c, int32_t nlayers, const int64_t* sizes, const int64_t* keep) {
+    if (!c) return SCALECOM_ERR_NULL_PTR;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;   // a step may still read the old table
+    if (nlayers == 0) {
+        cudaFree(c->layer_tab);
+        c->layer_tab = nullptr;
+        c->nlayers = 0;
+        return SCALECOM_OK;
+    }
+    if (nlayers < 0 || nlayers > int32_t(CS_MAX_LAYERS)) return SCALECOM_ERR_INVALID_ARG;
+    if (!sizes || !keep) return SCALECOM_ERR_NULL_PTR;
+    uint32_t* h = new (std::nothrow) uint32_t[2 * (size_t(nlayers) + 1)];
+    if (!h) return SCALECOM_ERR_ALLOC;
+    int64_t off = 0, ch = 0;
+    bool ok = true;
+    for (int32_t s = 0; s < nlayers && ok; ++s) {
+        ok = sizes[s] >= 1 && keep[s] >= 1 && keep[s] <= sizes[s] && sizes[s] <= c->d - off;
+        h[s] = uint32_t(off);
+        h[nlayers + 1 + s] = uint32_t(ch);
+        off += sizes[s];
+        ch += keep[s];
+    }
+    ok = ok && off == c->d && ch == c->k;
+    h[nlayers] = uint32_t(c->d);
+    h[2 * nlayers + 1] = uint32_t(c->k);
+    int rc = ok ? SCALECOM_OK : SCALECOM_ERR_INVALID_ARG;
+    if (ok) {
+        uint32_t* dev = nullptr;
+        const size_t bytes = 2 * (size_t(nlayers) + 1) * 4;
+        if (cudaMalloc(reinterpret_cast<void**>(&dev), bytes) != cudaSuccess) {
+            cudaGetLastError();
+            rc = SCALECOM_ERR_ALLOC;
+        } else if (cudaMemcpy(dev, h, bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(dev);
+            rc = SCALECOM_ERR_CUDA;
+        } else {
+            cudaFree(c->layer_tab);
+            c->layer_tab = dev;
+            c->nlayers = uint32_t(nlayers);
+        }
+    }
+    delete[] h;
+    return rc;
 }
 
 int scalecom_set_gathered(scalecom_ctx* c, float* dev_gathered) {
@@ -553,11 +609,11 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
             if (value == SCALECOM_SELECTOR_CHUNK && !c->chunk_best) {
                 DeviceGuard guard(c->device);
                 int occ = 0;
-                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, chunk_select_kernel<true>, CS_THREADS, 0) != cudaSuccess ||
+                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, chunk_select_kernel<true, true>, CS_THREADS, 0) != cudaSuccess ||
                     occ < 1)
                     return SCALECOM_ERR_CUDA;
                 if (occ > CS_BLOCKS_PER_SM) occ = CS_BLOCKS_PER_SM;
-                const int64_t per_block = int64_t(CS_THREADS / 32) * CS_GROUP;                 // chunks one block takes per round
+                const int64_t per_block = int64_t(CS_THREADS / 32) * CS_RUN;                   // chunks one block takes per round
                 const uint32_t need = uint32_t((c->k + per_block - 1) / per_block);
                 c->chunk_blocks = uint32_t(c->sms * occ) < need ? uint32_t(c->sms * occ) : need;
                 const size_t bytes = size_t(c->k) * 8;
@@ -566,7 +622,17 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
                     c->chunk_best = nullptr;
                     return SCALECOM_ERR_ALLOC;
                 }
-                if (cudaMemsetAsync(c->chunk_best, 0, bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+                const uint32_t one[4] = {0u, uint32_t(c->d), 0u, uint32_t(c->k)};
+                if (cudaMalloc(reinterpret_cast<void**>(&c->one_layer_tab), sizeof one) != cudaSuccess) {
+                    cudaGetLastError();
+                    cudaFree(c->chunk_best);
+                    c->chunk_best = nullptr;
+                    c->one_layer_tab = nullptr;
+                    return SCALECOM_ERR_ALLOC;
+                }
+                if (cudaMemsetAsync(c->chunk_best, 0, bytes, c->stream) != cudaSuccess ||
+                    cudaMemcpy(c->one_layer_tab, one, sizeof one, cudaMemcpyHostToDevice) != cudaSuccess)
+                    return SCALECOM_ERR_CUDA;
             }
             c->selector = int(value);
             return SCALECOM_OK;

@@ -187,3 +187,23 @@ def initial_weights(w: Workload, device) -> torch.Tensor:
 def initial_memory(w: Workload, device) -> List[torch.Tensor]:
     """Algorithm 1's input line: every learner's memory starts at zero."""
     return [torch.zeros(w.d, device=device, dtype=torch.float32) for _ in range(w.n)]
+
+
+def resnet50_layer_keep(w: Workload) -> Tuple[List[int], List[int]]:
+    """(sizes, keep) per tensor for the paper's per-layer rate rule (Section 4): 25X where a weight is
+    used in >= 196 multiply-adds per sample, 50X in [128, 196), 400X below, first convolution sent whole.
+    For an ImageNet ResNet-50 the uses per weight are the output positions of the layer: 112^2 for the
+    stem, 56^2 / 28^2 / 14^2 / 7^2 in the four stages, 1 for the classifier."""
+    segs = segments(w)
+    uses = [112 * 112] * 3                                   # stem conv + its two norm vectors
+    for width, blocks, hw in ((64, 3, 56), (128, 4, 28), (256, 6, 14), (512, 3, 7)):
+        for b in range(blocks):
+            uses += [hw * hw] * (9 + (3 if b == 0 else 0))
+    uses += [1, 1]
+    assert len(uses) == len(segs)
+    sizes, keep = [], []
+    for i, ((_, size), u) in enumerate(zip(segs, uses)):
+        rate = 1 if i == 0 else 25 if u >= 196 else 50 if u >= 128 else 400
+        sizes.append(size)
+        keep.append(max(1, size // rate))
+    return sizes, keep

@@ -42,7 +42,7 @@ def assert_step_matches(tag, idx_g, val_g, G_g, m_g, th_g, idx_o, val_o, G_o, m_
 
 
 def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exact=False, fuse_update=True,
-                    want_path=None, offset=0, use_hint=True, selector="topk", tag="case"):
+                    want_path=None, offset=0, use_hint=True, selector="topk", layers=None, tag="case"):
     """grads_per_step: list over steps of lists of n CUDA fp32 tensors.
     m0: list of n CUDA tensors (initial memory), theta0: CUDA tensor or None.
     offset > 0 places every device vector `offset` floats past a 16-byte boundary
@@ -72,6 +72,8 @@ def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exac
         ctx.set_option(binding.OPT_FUSE_UPDATE, int(fuse_update))
         ctx.set_option(binding.OPT_USE_HINT, int(use_hint))
         ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK if selector == "chunk" else binding.SELECTOR_TOPK)
+        if layers is not None:
+            ctx.set_layers(*layers)
         for s, grads in enumerate(grads_per_step):
             t = t0 + s
             g_dev = [place(g) for g in grads]
@@ -80,7 +82,7 @@ def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exac
             assert ctx.status() == 0, "%s step %d: device status %d" % (tag, s, ctx.status())
             paths.append(ctx.query(binding.Q_LAST_TOPK_PATH))
             g_np = [g.cpu().numpy() for g in grads]
-            idx_o, val_o, G_o = oracle.step(g_np, m_o, th_o, t, k, beta, lr, selector=selector)
+            idx_o, val_o, G_o = oracle.step(g_np, m_o, th_o, t, k, beta, lr, selector=selector, layers=layers)
             assert_step_matches("%s step %d" % (tag, s), idx.cpu().numpy(), val.cpu().numpy(),
                                 G.cpu().numpy().reshape(n, k), [x.cpu().numpy() for x in m_g],
                                 th_g.cpu().numpy() if th_g is not None else None,

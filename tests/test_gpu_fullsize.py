@@ -212,3 +212,13 @@ def test_maximum_dimension_chunk_selector():
     idx_o, _ = oracle.chunk_select(acc_h, k)
     assert np.array_equal(idx.cpu().numpy(), idx_o)
     assert np.array_equal(val.cpu().numpy(), acc_h[idx_o])
+
+
+def test_layer_rates_full_size_resnet50():
+    """Per-layer rates of Section 4 on the full ResNet-50-shaped vector, every element against the oracle."""
+    from tests.parity import workload_case
+    w = W.RESNET50
+    sizes, keep = W.resnet50_layer_keep(w)
+    w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
+    paths = workload_case(w2, 2, DEV, selector="chunk", layers=(sizes, keep))
+    assert paths == [3, 3]

@@ -383,3 +383,41 @@ def test_non_finite_inputs_follow_the_key_order(force_exact):
     for a, b in zip(md, m):
         assert np.array_equal(a.cpu().numpy(), b, equal_nan=True)
     assert np.array_equal(thd.cpu().numpy(), th, equal_nan=True)
+
+
+# ---- chunk-wise selector with per-layer rates (Section 4) ---------------------------------------------
+def test_layer_rates_small_cases():
+    rng = np.random.default_rng(31)
+    p = _parity()
+    for sizes, keep in [([7, 64, 1, 300, 128], [7, 2, 1, 3, 16]),
+                        ([5000], [50]),
+                        ([1] * 40, [1] * 40),
+                        ([1000, 3000, 2000, 4099], [1000, 30, 5, 4099])]:
+        d, k = sum(sizes), sum(keep)
+        g = [_t(rng.standard_normal(d)) for _ in range(3)]
+        m0 = [torch.zeros(d, device=DEV) for _ in range(3)]
+        paths = p.run_and_compare([g] * 3, m0, torch.linspace(-1, 1, d, device=DEV), k, 0.5, 0.25,
+                                  selector="chunk", layers=(sizes, keep), tag="layers %d" % len(sizes))
+        assert all(x == 3 for x in paths)
+
+
+def test_layer_rates_argument_checks():
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    with sc.Context(100, 2, 10, 0.5, 0.1) as ctx:
+        for sizes, keep in [([50, 49], [5, 5]), ([50, 50], [5, 4]), ([50, 50], [0, 10]), ([50, 50], [60, -50]), ([100] + [0], [10, 0])]:
+            with pytest.raises(sc.ScaleComError) as ei:
+                ctx.set_layers(sizes, keep)
+            assert ei.value.code == binding.ERR_INVALID_ARG
+        ctx.set_layers([50, 50], [5, 5])
+        ctx.set_layers(None)
+
+
+def test_layer_rates_resnet50_rule():
+    """The paper's rule on the ResNet-50-shaped workload at a test size: first tensor whole, 25X / 400X elsewhere."""
+    w = W.RESNET50.scaled(2_000_003)
+    sizes, keep = W.resnet50_layer_keep(w)
+    assert keep[0] == sizes[0] and len(sizes) == 161
+    w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
+    paths = _parity().workload_case(w2, 3, DEV, selector="chunk", layers=(sizes, keep))
+    assert all(x == 3 for x in paths)
