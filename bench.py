@@ -12,6 +12,7 @@ Rank 0 prints one JSON line.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import sys
@@ -48,6 +49,10 @@ def parse_args():
     ap.add_argument("--layers", action="store_true",
                     help="with --selector chunk on a ResNet-50-shaped workload: the paper's per-layer rate rule "
                          "(25X / 50X / 400X, first layer whole) instead of one rate; k becomes the sum of the layers' keeps")
+    ap.add_argument("--deployment", default="one-gpu", choices=["one-gpu", "learner-per-gpu"],
+                    help="one-gpu (default, the headline): all n learners of the workload in each GPU's memory; "
+                         "learner-per-gpu: every rank is one learner (n = number of ranks), indices broadcast and "
+                         "kept values all-gathered over NCCL between the library's calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -199,10 +204,111 @@ def time_oracle(w, batches_dev, steps=2, selector="topk", layers=None):
             "sample": "%d full steps of the bench workload (n=%d, d=%d, k=%d), %.1f s" % (steps, w.n, w.d, w.k, dt)}
 
 
+def run_learner_per_gpu(args):
+    """Every rank is one learner of Algorithm 1: select on the leader, index broadcast, compress, all-gather of
+    the kept values, reduce + weight update.  One JSON line from rank 0; the time is the max over ranks."""
+    import torch
+    import torch.distributed as dist
+    from paper_2104_11125_b200 import binding, multi, workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    else:
+        dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % (29400 + os.getpid() % 500),
+                                world_size=1, rank=0, device_id=dev)
+    w = dataclasses.replace(get_workload(args.workload), n=world)
+    K, Wm = args.steps, max(args.warmup, 3)
+    prof = W.profile(w, dev)
+    nb = max(1, min(K + Wm, args.batches, 4 * MAX_BATCHES))
+    grads = [W.gradients(w, s, dev, prof, learners=[rank])[0] for s in range(nb)]
+    mem = torch.zeros(w.d, device=dev, dtype=torch.float32)          # Algorithm 1: memory starts at zero
+    flush = torch.empty(64 << 20, device=dev, dtype=torch.float32)  # 256 MB: written between timed intervals
+    theta = W.initial_weights(w, dev)
+    node = multi.LearnerRank(w.d, w.k, w.beta, w.lr,
+                             selector=binding.SELECTOR_CHUNK if args.selector == "chunk" else binding.SELECTOR_TOPK)
+    ctx = node.engine
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    t = 0
+    for _ in range(Wm):
+        node.step(grads[t % nb], mem, theta, t)
+        t += 1
+    # the memory vector is the same 4d bytes every step and would sit in L2 from one step to the next, which a
+    # training iteration between two steps would not allow: each step is timed by itself, L2 flushed before it
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    launches0 = ctx.query(binding.Q_KERNEL_LAUNCHES)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    for a, b in evs:
+        flush.zero_()
+        a.record()
+        node.step(grads[t % nb], mem, theta, t)
+        b.record()
+        t += 1
+    barrier()
+    clocks = sampler.stop()
+    ms_step = sum(a.elapsed_time(b) for a, b in evs) / K
+    launches = ctx.query(binding.Q_KERNEL_LAUNCHES) - launches0
+    assert ctx.status() == 0, "device status %d" % ctx.status()
+
+    # the library's three calls one by one (CUDA events around each call, no collective in between)
+    def call_ms(fn, reps=30):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for i, (a, b) in enumerate(evs):
+            flush.zero_()
+            a.record()
+            fn(i)
+            b.record()
+        torch.cuda.synchronize()
+        ms = sorted(a.elapsed_time(b) for a, b in evs)
+        return ms[len(ms) // 2]
+
+    sel_ms = call_ms(lambda i: ctx.select(grads[i % nb], mem, node.idx))
+    cmp_ms = call_ms(lambda i: ctx.compress(grads[i % nb], mem, node.idx, node.own))
+    red_ms = call_ms(lambda i: ctx.reduce_rows(node.rows, node.val, node.idx, theta))
+    assert ctx.status() == 0
+    ms_step, sel_ms, cmp_ms, red_ms = max_over_ranks([ms_step, sel_ms, cmp_ms, red_ms], dev)
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        cmp_gbs = 12.0 * w.d / (cmp_ms * 1e-3) / 1e9
+        print(json.dumps({
+            "metric": METRIC, "value": world * w.d / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "n": world, "d": w.d, "k": w.k, "beta": w.beta, "lr": w.lr,
+                       "parallelism": "learner per GPU: index broadcast + all-gather of kept values (NCCL)",
+                       "selector": args.selector, "gradient_batches_resident": nb,
+                       "l2": "flushed (256 MB written) before every timed step and call",
+                       "exchange_bytes_per_rank_per_step": node.exchange_bytes()},
+            "roofline": {"bound": "hbm", "kernel": "scalecom_compress (index list -> bitmap, single-learner pass)",
+                         "achieved": cmp_gbs, "peak": peak, "unit": "GB/s", "frac": cmp_gbs / peak, "traffic": None,
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": 12.0 * w.d, "avg_launch_ms": cmp_ms},
+            "call_ms": {"scalecom_select": sel_ms, "scalecom_compress": cmp_ms, "scalecom_reduce_rows": red_ms,
+                        "note": "median of 30 calls, CUDA events around each call (about 6 us of event overhead each), L2 flushed before each"},
+            "gpu_launches": launches, "clocks": clocks,
+        }))
+    node.engine.close()
+    dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.deployment == "learner-per-gpu":
+        run_learner_per_gpu(args)
         return
 
     import torch

@@ -134,6 +134,37 @@ int scalecom_set_gathered(scalecom_ctx* ctx, float* dev_gathered);
 int scalecom_set_layers(scalecom_ctx* ctx, int32_t nlayers, const int64_t* sizes, const int64_t* keep);
 
 /*
+ * The step taken apart, for the learner-per-GPU deployment the paper describes (Section 4, Appendix E:
+ * the leading worker's indices are broadcast, every worker compresses its own error-feedback gradient
+ * with them, the kept values are reduced across workers).  One handle per rank, created with the
+ * global d and k; the collectives between the three calls are the caller's (NCCL or any other):
+ *
+ *   leader rank (t mod world):   scalecom_select(g, m, idx)                          step 2
+ *   all ranks, after the broadcast of idx:
+ *                                scalecom_compress(g, m, idx, gathered)              steps 1, 3 (gather), 4
+ *   all ranks, after an all-gather of the `gathered` rows into rows[world][k] (rank order):
+ *                                scalecom_reduce_rows(rows, world, val, idx, theta)  step 3 (reduce) and step 5
+ *
+ * Summing the gathered rows locally in rank order (k values per rank cross the links, as in the paper)
+ * keeps the result identical, bit for bit, to scalecom_step on one GPU holding all the learners.
+ * All pointers DEVICE; all three calls are asynchronous on the handle's stream.
+ *   scalecom_select    g, m fp32[d] read only; out_idx int32[k] written, ascending (selector as set by
+ *                      SCALECOM_OPT_SELECTOR).
+ *   scalecom_compress  g fp32[d] read only; m fp32[d] updated in place (Eq. 4); idx int32[k] strictly
+ *                      ascending, < d (otherwise scalecom_status reports INTERNAL and nothing is written
+ *                      out of bounds); out_gathered fp32[k] = (m + g)[idx[j]] written.
+ *   scalecom_reduce_rows  rows fp32[n_rows * k] read only; out_val fp32[k] = (sum over rows, in order) / n_rows
+ *                      written.  weights fp32[d], if not NULL, gets Algorithm 1 line 12 in the same kernel:
+ *                      weights[idx[j]] -= lr * out_val[j], with idx int32[k] the broadcast list (an entry >= d
+ *                      is skipped and scalecom_status reports INTERNAL); weights NULL: no update, idx unused.
+ * Errors (all three): NULL_PTR, ALIAS, BAD_STATE, ALLOC (compress, first call), CUDA; INVALID_ARG for n_rows < 1.
+ */
+int scalecom_select(scalecom_ctx* ctx, const float* g, const float* m, int32_t* out_idx);
+int scalecom_compress(scalecom_ctx* ctx, const float* g, float* m, const int32_t* idx, float* out_gathered);
+int scalecom_reduce_rows(scalecom_ctx* ctx, const float* rows, int32_t n_rows, float* out_val, const int32_t* idx,
+                         float* weights);
+
+/*
  * Algorithm 1 line 12 on its own: theta[idx[j]] <- theta[idx[j]] - lr * val[j]
  * for j < k, on the handle's stream, for callers that ran scalecom_step with
  * weights == NULL.  All pointers DEVICE; idx entries must be distinct and < d.

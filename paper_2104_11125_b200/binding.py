@@ -31,7 +31,7 @@ EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
     "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
-    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance", "scalecom_set_layers",
+    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance", "scalecom_set_layers", "scalecom_select", "scalecom_compress", "scalecom_reduce_rows",
 )
 STATIC_MAX_D = 1 << 20
 
@@ -88,6 +88,12 @@ def lib() -> ctypes.CDLL:
         L.scalecom_cosine_distance.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_double)]
         L.scalecom_set_layers.restype = ctypes.c_int
         L.scalecom_set_layers.argtypes = [vp, i32, vp, vp]
+        L.scalecom_select.restype = ctypes.c_int
+        L.scalecom_select.argtypes = [vp, vp, vp, vp]
+        L.scalecom_compress.restype = ctypes.c_int
+        L.scalecom_compress.argtypes = [vp, vp, vp, vp, vp]
+        L.scalecom_reduce_rows.restype = ctypes.c_int
+        L.scalecom_reduce_rows.argtypes = [vp, vp, i32, vp, vp, vp]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -160,8 +166,9 @@ class Context:
 
     def close(self) -> None:
         if getattr(self, "_h", None):
-            scalecom_destroy(self._h)
-            self._h = None
+            h, self._h = self._h, None
+            if _lib is not None:                 # at interpreter exit the module globals may already be gone
+                _lib.scalecom_destroy(h)
 
     __del__ = close
 
@@ -219,6 +226,29 @@ class Context:
         kp = (ctypes.c_int64 * len(keep))(*[int(x) for x in keep])
         _check(lib().scalecom_set_layers(self._h, len(sizes), ctypes.cast(sz, ctypes.c_void_p),
                                          ctypes.cast(kp, ctypes.c_void_p)), "scalecom_set_layers")
+
+    def _idx(self, idx: torch.Tensor) -> int:
+        if not (idx.is_cuda and idx.dtype == torch.int32 and idx.is_contiguous() and idx.numel() == self.k):
+            raise TypeError("idx must be a contiguous CUDA int32 tensor of k elements")
+        return idx.data_ptr()
+
+    def select(self, g: torch.Tensor, m: torch.Tensor, out_idx: torch.Tensor) -> None:
+        _check(lib().scalecom_select(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"), self._idx(out_idx)),
+               "scalecom_select")
+
+    def compress(self, g: torch.Tensor, m: torch.Tensor, idx: torch.Tensor, out_gathered: torch.Tensor) -> None:
+        _check(lib().scalecom_compress(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"), self._idx(idx),
+                                       _dev_f32(out_gathered, self.k, "out_gathered")), "scalecom_compress")
+
+    def reduce_rows(self, rows: torch.Tensor, out_val: torch.Tensor, idx: Optional[torch.Tensor] = None,
+                    weights: Optional[torch.Tensor] = None) -> None:
+        """out_val = mean of the rows in row order; with idx and weights also weights[idx] -= lr * out_val."""
+        n_rows = max(1, rows.numel() // self.k)
+        _check(lib().scalecom_reduce_rows(self._h, _dev_f32(rows, n_rows * self.k, "rows"), n_rows,
+                                          _dev_f32(out_val, self.k, "out_val"),
+                                          None if idx is None else self._idx(idx),
+                                          None if weights is None else _dev_f32(weights, self.d, "weights")),
+               "scalecom_reduce_rows")
 
     def overlap(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], t: int) -> int:
         """Eq. 5's d between the leader's top-k set and the true top-k set (synchronous)."""

@@ -23,6 +23,14 @@ namespace sc {
 constexpr int LP_THREADS = 256;            // x 4 coordinates = one tile
 constexpr int LP_UNROLL = SC_LP_UNROLL;    // learners in flight per thread
 constexpr int LP_BLOCKS_PER_SM = SC_LP_BLOCKS_PER_SM;
+#ifndef SC_ONE_T
+#define SC_ONE_T 2
+#endif
+#ifndef SC_ONE_BLOCKS
+#define SC_ONE_BLOCKS 4
+#endif
+constexpr int LP_ONE_T = SC_ONE_T;                 // tiles per burst of the single-learner form
+constexpr int LP_ONE_BLOCKS_PER_SM = SC_ONE_BLOCKS;
 
 template <int N>
 struct PtrTable {
@@ -35,6 +43,7 @@ struct LearnerParams {
     int32_t n;
     float beta, omb, lr, nf;               // omb = 1 - beta rounded once in fp32; nf = (float)n
     const uint32_t* bitmap;                // [ntiles * 32]
+    uint32_t* bitmap_clear;                // single-learner form: the same words, zeroed once read (or nullptr)
     const uint32_t* tile_prefix;           // [ntiles + 1]
     float* out_val;                        // [k]
     int32_t* out_idx;                      // [k]: the ascending index list, written here from the ranks
@@ -46,46 +55,39 @@ struct LearnerParams {
 // One burst of a thread covers LP_T consecutive tiles x LP_L learners (LP_T * LP_L = LP_UNROLL pairs of
 // 128-bit loads in flight).  Few learners: more tiles per burst keep the loads in flight; many
 // learners: fewer arrays per burst keep each burst inside a few pages.
-template <int N, bool VEC, int LP_T, int LP_L>
-__global__ void __launch_bounds__(LP_THREADS, LP_BLOCKS_PER_SM)
+// ONE: the single-learner form used when every learner has its own device -- n is 1 at compile time, no
+// weights are touched (the reduced values do not exist yet), and ranks are checked against k before a value
+// is written, because the bitmap and prefix counts then come from an index list received from elsewhere.
+template <int N, bool VEC, int LP_T, int LP_L, bool ONE = false>
+__global__ void __launch_bounds__(LP_THREADS, ONE ? LP_ONE_BLOCKS_PER_SM : LP_BLOCKS_PER_SM)
 learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P) {
-    static_assert(LP_T * LP_L == LP_UNROLL, "burst shape");
+    static_assert(LP_T * LP_L <= LP_UNROLL, "burst shape");
+    constexpr bool GUARD = ONE;
     const uint32_t tid = threadIdx.x, lane = lane_id();
     const uint32_t d = P.d;
-    const int n = P.n;
+    const int n = ONE ? 1 : P.n;
+    float* const weights = ONE ? nullptr : P.weights;
+    float* const gathered = ONE ? nullptr : P.gathered;
     const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside a tile
     const uint32_t sh = (tid & 7u) * 4u;           // and its first bit inside that word
     span_begin(P.spans);
 
     const uint32_t nsuper = (P.ntiles + LP_T - 1) / LP_T;
     for (uint32_t sup = blockIdx.x; sup < nsuper; sup += gridDim.x) {
-        // per tile: selection bits of this thread's four coordinates and the rank of the first selected one
-        uint32_t nib[LP_T], rank0[LP_T], pc[LP_T];
+        // Single-learner form: the first (only) burst of g and m is requested before anything waits on the
+        // bitmap, so that one memory latency covers both.  With several learners per tile the later order
+        // measured faster (the loads of a burst then issue back to back with nothing else in flight).
+        uint32_t pc[LP_T], bw[LP_T], tp[LP_T];
 #pragma unroll
         for (int t = 0; t < LP_T; ++t) {
             const uint32_t tile = sup * LP_T + t;
             const bool have = tile < P.ntiles;                         // uniform across the block
-            const uint32_t w = have ? __ldg(&P.bitmap[size_t(tile) * 32 + lane]) : 0u;
-            const uint32_t cnt = __popc(w);
-            const uint32_t incl = warp_incl_scan(cnt);
-            const uint32_t excl_word = __shfl_sync(FULL, incl - cnt, wi);
-            const uint32_t myword = __shfl_sync(FULL, w, wi);
-            nib[t] = (myword >> sh) & 15u;
-            rank0[t] = (have ? __ldg(&P.tile_prefix[tile]) : 0u) + excl_word + __popc(myword & ((1u << sh) - 1u));
             pc[t] = have ? tile * TILE + tid * 4u : d;                 // d: nothing to do
+            bw[t] = !have ? 0u : ONE ? P.bitmap[size_t(tile) * 32 + lane] : __ldg(&P.bitmap[size_t(tile) * 32 + lane]);
+            tp[t] = have ? __ldg(&P.tile_prefix[tile]) : 0u;
         }
-
-        // weights at the selected coordinates, fetched now so that their latency hides behind the learner loop
-        float wv[LP_T][4];
-#pragma unroll
-        for (int t = 0; t < LP_T; ++t)
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                wv[t][c] = (P.weights && ((nib[t] >> c) & 1u) && pc[t] + c < d) ? P.weights[pc[t] + c] : 0.0f;
-
-        float sum[LP_T][4];
-        for (int i0 = 0; i0 < n; i0 += LP_L) {
-            float gv[LP_T][LP_L][4], mv[LP_T][LP_L][4];
+        float gv[LP_T][LP_L][4], mv[LP_T][LP_L][4];
+        auto load_burst = [&](int i0) {
 #pragma unroll
             for (int t = 0; t < LP_T; ++t)
 #pragma unroll
@@ -94,6 +96,41 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                         load_quad_stream<VEC>(tab.g[i0 + u], pc[t], d, gv[t][u]);
                         load_quad_stream<VEC>(tab.m[i0 + u], pc[t], d, mv[t][u]);
                     }
+        };
+        if (ONE) load_burst(0);
+
+        // per tile: selection bits of this thread's four coordinates and the rank of the first selected one
+        uint32_t nib[LP_T], rank0[LP_T];
+#pragma unroll
+        for (int t = 0; t < LP_T; ++t) {
+            const uint32_t cnt = __popc(bw[t]);
+            const uint32_t incl = warp_incl_scan(cnt);
+            const uint32_t excl_word = __shfl_sync(FULL, incl - cnt, wi);
+            const uint32_t myword = __shfl_sync(FULL, bw[t], wi);
+            nib[t] = (myword >> sh) & 15u;
+            rank0[t] = tp[t] + excl_word + __popc(myword & ((1u << sh) - 1u));
+        }
+
+        if (ONE && P.bitmap_clear) {           // every warp has its copy of the words: leave the bitmap zero for the next list
+            __syncthreads();
+            if (tid < 32) {
+#pragma unroll
+                for (int t = 0; t < LP_T; ++t)
+                    if (sup * LP_T + t < P.ntiles) P.bitmap_clear[size_t(sup * LP_T + t) * 32 + lane] = 0u;
+            }
+        }
+
+        // weights at the selected coordinates, fetched now so that their latency hides behind the learner loop
+        float wv[LP_T][4];
+#pragma unroll
+        for (int t = 0; t < LP_T; ++t)
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                wv[t][c] = (weights && ((nib[t] >> c) & 1u) && pc[t] + c < d) ? weights[pc[t] + c] : 0.0f;
+
+        float sum[LP_T][4];
+        for (int i0 = 0; i0 < n; i0 += LP_L) {
+            if (!ONE || i0 > 0) load_burst(i0);
 #pragma unroll
             for (int t = 0; t < LP_T; ++t)
 #pragma unroll
@@ -109,11 +146,11 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                             out[c] = __fadd_rn(__fmul_rn(P.omb, mv[t][u][c]), __fmul_rn(P.beta, r));   // Eq. 4
                         }
                         store_quad_stream<VEC>(tab.m[i], pc[t], d, out);
-                        if (nib[t] && P.gathered) {                                           // Eq. 3: learner i's kept values
+                        if (nib[t] && gathered) {                                             // Eq. 3: learner i's kept values
                             uint32_t r = rank0[t];
 #pragma unroll
                             for (int c = 0; c < 4; ++c)
-                                if ((nib[t] >> c) & 1u) P.gathered[size_t(i) * P.k + r++] = acc[c];
+                                if (((nib[t] >> c) & 1u) && (!GUARD || r < P.k)) gathered[size_t(i) * P.k + r++] = acc[c];
                         }
                     }
         }
@@ -123,11 +160,11 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                 uint32_t r = rank0[t];
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    if ((nib[t] >> c) & 1u) {
+                    if (((nib[t] >> c) & 1u) && (!GUARD || r < P.k)) {
                         const float v = __fdiv_rn(sum[t][c], P.nf);                           // line 10: one division by n
                         P.out_idx[r] = int32_t(pc[t] + c);
                         P.out_val[r++] = v;
-                        if (P.weights) P.weights[pc[t] + c] = __fsub_rn(wv[t][c], __fmul_rn(P.lr, v));   // line 12
+                        if (weights) weights[pc[t] + c] = __fsub_rn(wv[t][c], __fmul_rn(P.lr, v));   // line 12
                     }
             }
     }

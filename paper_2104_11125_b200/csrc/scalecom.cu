@@ -11,6 +11,7 @@
 
 #include "chunk_select.cuh"
 #include "diagnostics.cuh"
+#include "exchange.cuh"
 #include "learner_pass.cuh"
 #include "topk_select.cuh"
 
@@ -37,7 +38,7 @@ struct scalecom_ctx {
     // launch geometry
     int sms = 0;
     uint32_t topk_blocks = 0, lp_blocks = 0;
-    int lp_tiles = 1;                  // tiles per burst of the learner pass
+    mutable bool bitmap_zero = false;  // the bitmap holds no bits (scalecom_compress leaves it so; selection kernels do not)
     uint32_t samp_stride = 1, samp_target = 1;
 
     // options
@@ -76,6 +77,8 @@ struct scalecom_ctx {
     float* diag_zero = nullptr;        // [d], all zero
     uint32_t* diag_bitmap = nullptr;   // [ntiles * 32]
     double* diag_acc = nullptr;        // [4]: overlap count (as u64) and three dot products
+
+    int32_t* scratch_idx = nullptr;    // [k] index list the learner pass writes when the caller already has one
 };
 
 namespace {
@@ -98,6 +101,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 template <bool VEC>
 cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
+    c->bitmap_zero = false;
     void* args[] = {const_cast<TopkParams*>(&P)};
     return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&topk_select_kernel<VEC>), dim3(c->topk_blocks),
                                        dim3(TK_THREADS), args, sizeof(TopkShared), c->stream);
@@ -105,44 +109,52 @@ cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
 
 template <bool VEC>
 cudaError_t launch_chunk(const scalecom_ctx* c, const ChunkParams& P) {
+    c->bitmap_zero = false;
     void* args[] = {const_cast<ChunkParams*>(&P)};
     const void* fn = P.nl > 1 ? reinterpret_cast<const void*>(&chunk_select_kernel<VEC, true>)
                               : reinterpret_cast<const void*>(&chunk_select_kernel<VEC, false>);
     return cudaLaunchCooperativeKernel(fn, dim3(c->chunk_blocks), dim3(CS_THREADS), args, 0, c->stream);
 }
 
-template <int N, bool VEC, int T>
-cudaError_t launch_learner(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
+template <int N, bool VEC, int T, int L = LP_UNROLL / T, bool ONE = false>
+cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem, const LearnerParams& P) {
     PtrTable<N> tab;
     for (int i = 0; i < N; ++i) {
-        tab.g[i] = i < c->n ? grads[i] : nullptr;
-        tab.m[i] = i < c->n ? mem[i] : nullptr;
+        tab.g[i] = i < n ? grads[i] : nullptr;
+        tab.m[i] = i < n ? mem[i] : nullptr;
     }
     const uint32_t nsuper = (c->ntiles + T - 1) / T;
-    const uint32_t blocks = c->lp_blocks < nsuper ? c->lp_blocks : nsuper;
-    learner_pass_kernel<N, VEC, T, LP_UNROLL / T><<<blocks, LP_THREADS, 0, c->stream>>>(tab, P);
+    const uint32_t want = ONE ? uint32_t(c->sms) * LP_ONE_BLOCKS_PER_SM : c->lp_blocks;
+    const uint32_t blocks = want < nsuper ? want : nsuper;
+    learner_pass_kernel<N, VEC, T, L, ONE><<<blocks, LP_THREADS, 0, c->stream>>>(tab, P);
     return cudaGetLastError();
 }
 
-// burst shape (tiles x learners) by learner count
+// burst shape (tiles x learners) by learner count: few learners take more tiles per burst
+inline int burst_tiles(int n) { return n >= 8 ? 1 : n >= 4 ? 2 : n >= 2 ? 4 : 0; }
+
 template <int N, bool VEC>
-cudaError_t launch_learner_t(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
-    switch (c->lp_tiles) {
-        case 1: return launch_learner<N, VEC, 1>(c, grads, mem, P);
-        case 2: return launch_learner<N, VEC, 2>(c, grads, mem, P);
-        case 4: return launch_learner<N, VEC, 4>(c, grads, mem, P);
-        default: return launch_learner<N, VEC, 8>(c, grads, mem, P);
+cudaError_t launch_learner_t(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem,
+                             const LearnerParams& P) {
+    switch (burst_tiles(n)) {
+        case 1: return launch_learner<N, VEC, 1>(c, n, grads, mem, P);
+        case 2: return launch_learner<N, VEC, 2>(c, n, grads, mem, P);
+        case 4: return launch_learner<N, VEC, 4>(c, n, grads, mem, P);
+        default: return launch_learner<N, VEC, 4, 1>(c, n, grads, mem, P);   // one learner: 8 tiles per burst spill
     }
 }
 
+// n learners of the caller's tables through the learner pass (n may be less than the handle's)
 template <bool VEC>
-cudaError_t launch_learner_n(const scalecom_ctx* c, const float* const* grads, float* const* mem, const LearnerParams& P) {
-    if (c->n <= 16) return launch_learner_t<16, VEC>(c, grads, mem, P);
-    if (c->n <= 128) return launch_learner_t<128, VEC>(c, grads, mem, P);
-    return launch_learner_t<SCALECOM_MAX_LEARNERS, VEC>(c, grads, mem, P);
+cudaError_t launch_learner_n(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem,
+                             const LearnerParams& P) {
+    if (n <= 16) return launch_learner_t<16, VEC>(c, n, grads, mem, P);
+    if (n <= 128) return launch_learner_t<128, VEC>(c, n, grads, mem, P);
+    return launch_learner_t<SCALECOM_MAX_LEARNERS, VEC>(c, n, grads, mem, P);
 }
 
 int init_workspace(scalecom_ctx* c) {
+    c->bitmap_zero = false;
     if (cudaMemsetAsync(c->ws, 0, c->ctrl_region_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     if (c->chunk_best && cudaMemsetAsync(c->chunk_best, 0, size_t(c->k) * 8, c->stream) != cudaSuccess)
         return SCALECOM_ERR_CUDA;
@@ -222,7 +234,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     lp.omb = 1.0f - c->beta;
     lp.lr = c->lr;
     lp.nf = float(c->n);
-    lp.bitmap = c->bitmap;
+    lp.bitmap = c->bitmap; lp.bitmap_clear = nullptr;
     lp.tile_prefix = c->tile_prefix;
     lp.out_val = out_val;
     lp.out_idx = out_idx;
@@ -259,7 +271,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     if (tm && cudaEventRecord(ev[1], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
-    e = vec_all ? launch_learner_n<true>(c, grads, mem, lp) : launch_learner_n<false>(c, grads, mem, lp);
+    e = vec_all ? launch_learner_n<true>(c, c->n, grads, mem, lp) : launch_learner_n<false>(c, c->n, grads, mem, lp);
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     if (tm && cudaEventRecord(ev[2], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
@@ -327,7 +339,6 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->tiles_per_block = (c->ntiles + c->topk_blocks - 1) / c->topk_blocks;
     c->lp_blocks = uint32_t(c->sms * occ_lp);
     if (c->lp_blocks > c->ntiles) c->lp_blocks = c->ntiles;
-    c->lp_tiles = n >= 8 ? 1 : n >= 4 ? 2 : n >= 2 ? 4 : 8;
 
     // sampling rate: about 2^18 sampled keys or 1/64 of the vector, whichever is more
     uint32_t stride = 1;
@@ -465,6 +476,7 @@ void scalecom_destroy(scalecom_ctx* c) {
     cudaFree(c->diag_zero);
     cudaFree(c->diag_bitmap);
     cudaFree(c->diag_acc);
+    cudaFree(c->scratch_idx);
     cudaFree(c->stage_g);
     cudaFree(c->stage_idx);
     cudaFree(c->stage_val);
@@ -541,6 +553,98 @@ int scalecom_apply_update(scalecom_ctx* c, float* weights, const int32_t* idx, c
     if (!guard.ok) return SCALECOM_ERR_CUDA;
     const uint32_t blocks = uint32_t((k + 255) / 256);
     apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, idx, val, uint32_t(k), lr);
+    if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+    ++c->launches;
+    return SCALECOM_OK;
+}
+
+int scalecom_select(scalecom_ctx* c, const float* g, const float* m, int32_t* out_idx) {
+    if (!c || !g || !m || !out_idx) return SCALECOM_ERR_NULL_PTR;
+    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    const bool vec = aligned16(g) && aligned16(m);
+    cudaError_t e;
+    if (c->selector == SCALECOM_SELECTOR_CHUNK) {
+        ChunkParams cp;
+        cp.g = g; cp.m = m; cp.d = uint32_t(c->d); cp.k = uint32_t(c->k);
+        cp.spin_limit = c->spin_limit;
+        cp.best = c->chunk_best;
+        cp.bitmap = c->bitmap; cp.tile_prefix = c->tile_prefix; cp.ntiles = c->ntiles;
+        cp.ctrl = c->ctrl;
+        cp.barrier = c->barrier + 8;
+        cp.out_idx = out_idx;
+        cp.spans = nullptr;
+        cp.nl = c->nlayers ? c->nlayers : 1u;
+        cp.layer_off = c->nlayers ? c->layer_tab : c->one_layer_tab;
+        cp.layer_chunk0 = cp.layer_off + (cp.nl + 1);
+        e = vec ? launch_chunk<true>(c, cp) : launch_chunk<false>(c, cp);
+    } else {
+        // one vector, one hint slot: the handle of a learner-per-GPU rank always sees the same learner
+        TopkParams tp = make_topk_params(c, g, m, c->leader_hint, true, nullptr);
+        tp.out_idx = out_idx;
+        e = vec ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
+    }
+    if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
+    ++c->launches;
+    return SCALECOM_OK;
+}
+
+int scalecom_compress(scalecom_ctx* c, const float* g, float* m, const int32_t* idx, float* out_gathered) {
+    if (!c || !g || !m || !idx || !out_gathered) return SCALECOM_ERR_NULL_PTR;
+    if (static_cast<const void*>(g) == static_cast<const void*>(m) || static_cast<const void*>(idx) == out_gathered)
+        return SCALECOM_ERR_ALIAS;
+    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    if (!c->scratch_idx && cudaMalloc(reinterpret_cast<void**>(&c->scratch_idx), size_t(c->k) * 4) != cudaSuccess) {
+        cudaGetLastError();
+        c->scratch_idx = nullptr;
+        return SCALECOM_ERR_ALLOC;
+    }
+    // the received index list -> bitmap and tile prefixes in the handle's workspace
+    // (the single-learner pass below zeroes every bitmap word it has read, so only a bitmap that a selection
+    // kernel wrote since, or a fresh workspace, has to be cleared here)
+    if (!c->bitmap_zero &&
+        cudaMemsetAsync(c->bitmap, 0, size_t(c->ntiles) * 32 * 4, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    c->bitmap_zero = true;
+    const uint32_t for_idx = uint32_t((c->k + 255) / 256), for_tiles = c->ntiles / 8 + 1, cap = uint32_t(c->sms) * 16u;
+    const uint32_t want = for_idx > for_tiles ? for_idx : for_tiles;
+    indices_to_bitmap_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(idx, uint32_t(c->k), uint32_t(c->d), c->ntiles,
+                                                                            c->bitmap, c->tile_prefix, c->ctrl + CT_STATUS);
+    if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+    // this learner's share of steps 1, 3 and 4: a learner pass over one learner; with n = 1 the
+    // "average" it writes is the gathered value itself (x / 1 is exact)
+    LearnerParams lp;
+    lp.d = uint32_t(c->d); lp.k = uint32_t(c->k); lp.ntiles = c->ntiles;
+    lp.n = 1;
+    lp.beta = c->beta; lp.omb = 1.0f - c->beta; lp.lr = c->lr; lp.nf = 1.0f;
+    lp.bitmap = c->bitmap; lp.bitmap_clear = c->bitmap; lp.tile_prefix = c->tile_prefix;
+    lp.out_val = out_gathered; lp.out_idx = c->scratch_idx;
+    lp.gathered = nullptr; lp.weights = nullptr; lp.spans = nullptr;
+    const float* gp[1] = {g};
+    float* mp[1] = {m};
+    const cudaError_t e = (aligned16(g) && aligned16(m)) ? launch_learner<16, true, LP_ONE_T, 1, true>(c, 1, gp, mp, lp)
+                                                         : launch_learner<16, false, LP_ONE_T, 1, true>(c, 1, gp, mp, lp);
+    if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
+    c->launches += 2;
+    return SCALECOM_OK;
+}
+
+int scalecom_reduce_rows(scalecom_ctx* c, const float* rows, int32_t n_rows, float* out_val, const int32_t* idx,
+                         float* weights) {
+    if (!c || !rows || !out_val || (weights && !idx)) return SCALECOM_ERR_NULL_PTR;
+    if (n_rows < 1) return SCALECOM_ERR_INVALID_ARG;
+    if (static_cast<const void*>(rows) == out_val || static_cast<const void*>(weights) == out_val ||
+        static_cast<const void*>(weights) == rows || static_cast<const void*>(idx) == out_val)
+        return SCALECOM_ERR_ALIAS;
+    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    const uint32_t want = uint32_t((c->k + 255) / 256), cap = uint32_t(c->sms) * 8u;
+    reduce_rows_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(rows, n_rows, uint32_t(c->k), float(n_rows), out_val,
+                                                                      idx, weights, uint32_t(c->d), c->lr,
+                                                                      c->ctrl + CT_STATUS);
     if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     return SCALECOM_OK;

@@ -1,0 +1,88 @@
+"""One rank of a learner-per-process job, run as a child process by test_exchange.py.
+
+usage: exchange_worker.py <cpu|gpu> <topk|chunk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
+
+Every rank generates all learners' seeded inputs, takes the learner of its own rank through
+multi.LearnerRank, and checks each step's index list, reduced values, its learner's memory and
+its weight replica, bit for bit, against the oracle's single-process step over all learners.
+
+"gpu": the library's kernels on cuda:0 (the ranks share the device; nothing in a kernel waits for
+another rank, the exchanges are gloo collectives between launches).
+"cpu": the same orchestration over an engine made of the oracle's pieces, so that leader rotation,
+broadcast source and row order are checked where there is no GPU.
+"""
+import os
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+import oracle  # noqa: E402
+from paper_2104_11125_b200 import binding, multi, workloads  # noqa: E402
+
+
+class OracleEngine:
+    """Test-only stand-in with the three calls LearnerRank makes, on CPU tensors."""
+
+    def __init__(self, d, k, beta, lr, selector):
+        self.d, self.k, self.beta, self.lr, self.selector = d, k, beta, lr, selector
+
+    def select(self, g, m, out_idx):
+        acc = oracle.accumulate(g.numpy(), m.numpy())
+        idx, _ = (oracle.chunk_select if self.selector == "chunk" else oracle.topk)(acc, self.k)
+        out_idx.copy_(torch.from_numpy(idx))
+
+    def compress(self, g, m, idx, out):
+        sel = np.zeros(self.d, np.uint8)
+        sel[idx.numpy()] = 1
+        out.copy_(torch.from_numpy(oracle.learner(g.numpy(), m.numpy(), idx.numpy(), sel, self.beta)))
+
+    def reduce_rows(self, rows, val, idx=None, weights=None):
+        val.copy_(torch.from_numpy(oracle.reduce(rows.view(-1, self.k).numpy())))
+        if weights is not None:
+            oracle.apply(weights.numpy(), idx.numpy(), val.numpy(), self.lr)
+
+
+def main():
+    mode, selector, d, steps = sys.argv[1], sys.argv[2], int(sys.argv[3]), int(sys.argv[4])
+    dist.init_process_group("gloo")
+    rank, world = dist.get_rank(), dist.get_world_size()
+    w = workloads.TINY.scaled(d, world)
+    k, beta, lr = w.k, w.beta, w.lr
+    dev = torch.device("cuda", 0) if mode == "gpu" else torch.device("cpu")
+    if mode == "gpu":
+        torch.cuda.set_device(dev)
+        node = multi.LearnerRank(d, k, beta, lr,
+                                 selector=binding.SELECTOR_CHUNK if selector == "chunk" else binding.SELECTOR_TOPK)
+    else:
+        node = multi.LearnerRank(d, k, beta, lr, engine=OracleEngine(d, k, beta, lr, selector), device=dev)
+    prof = workloads.profile(w, dev)
+    m_o = [x.cpu().numpy().copy() for x in workloads.initial_memory(w, dev)]
+    th_o = workloads.initial_weights(w, dev).cpu().numpy().copy()
+    mem = torch.from_numpy(m_o[rank].copy()).to(dev)
+    theta = torch.from_numpy(th_o.copy()).to(dev)
+    for t in range(steps):
+        g_dev = workloads.gradients(w, t, dev, prof)
+        g_all = [g.cpu().numpy() for g in g_dev]
+        grad = g_dev[rank].contiguous()
+        idx, val = node.step(grad, mem, theta, t)
+        if mode == "gpu":
+            torch.cuda.synchronize()
+            assert node.engine.status() == binding.OK
+        idx_o, val_o, _ = oracle.step(g_all, m_o, th_o, t, k, beta, lr, want_gathered=False, selector=selector)
+        assert np.array_equal(idx.cpu().numpy(), idx_o), "step %d rank %d: index lists differ" % (t, rank)
+        assert np.array_equal(val.cpu().numpy(), val_o), "step %d rank %d: reduced values differ" % (t, rank)
+        assert np.array_equal(mem.cpu().numpy(), m_o[rank]), "step %d rank %d: memory differs" % (t, rank)
+        assert np.array_equal(theta.cpu().numpy(), th_o), "step %d rank %d: weights differ" % (t, rank)
+    assert node.exchange_bytes() == (4 * k * world if world > 1 else 0)
+    dist.barrier()
+    dist.destroy_process_group()
+    print("rank", rank, "ok")
+
+
+if __name__ == "__main__":
+    main()

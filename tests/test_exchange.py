@@ -1,0 +1,164 @@
+"""Learner-per-process deployment (one learner per rank, index broadcast + all-gather of the kept
+values): every rank must reproduce, bit for bit, the single-process step of Algorithm 1 over the
+same learners.  The ranks are child processes joined over gloo on 127.0.0.1."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+WORKER = os.path.join(HERE, "exchange_worker.py")
+
+
+def run_ranks(world, mode, selector, d, steps, timeout=240):
+    port = 23000 + (os.getpid() * 7 + world * 13 + len(selector)) % 4000
+    procs = []
+    for rank in range(world):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, WORKER, mode, selector, str(d), str(steps)], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
+    outs = []
+    try:
+        for p in procs:
+            out, _ = p.communicate(timeout=timeout)
+            outs.append(out)
+    finally:
+        for p in procs:
+            if p.poll() is None:
+                p.kill()
+    for rank, (p, out) in enumerate(zip(procs, outs)):
+        assert p.returncode == 0, "rank %d:\n%s" % (rank, out[-3000:])
+        assert "rank %d ok" % rank in out
+
+
+@pytest.mark.parametrize("world,selector", [(2, "topk"), (3, "topk"), (2, "chunk")])
+def test_protocol_over_gloo_matches_single_process_step(world, selector):
+    # 2 * world + 1 steps: every rank leads at least twice
+    run_ranks(world, "cpu", selector, 40_003, 2 * world + 1)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("world,selector,d", [(2, "topk", 262_147), (3, "topk", 1_048_583), (3, "chunk", 262_147)])
+def test_ranks_sharing_a_device_match_single_process_step(world, selector, d):
+    run_ranks(world, "gpu", selector, d, 2 * world + 1, timeout=400)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("selector,d,n", [("topk", 300_007, 4), ("chunk", 300_007, 4), ("topk", 5_000_011, 5)])
+def test_pieces_in_one_process_match_oracle_step(selector, d, n):
+    """The calls of the taken-apart step, one handle per learner, without any collective."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2104_11125_b200 import binding, workloads
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    w = workloads.TINY.scaled(d, n)
+    k, beta, lr = w.k, w.beta, w.lr
+    prof = workloads.profile(w, dev)
+    mem = workloads.initial_memory(w, dev)
+    m_o = [x.cpu().numpy().copy() for x in mem]
+    theta = [workloads.initial_weights(w, dev) for _ in range(n)]
+    th_o = theta[0].cpu().numpy().copy()
+    ctxs = [sc.Context(d, 1, k, beta, lr) for _ in range(n)]
+    for c in ctxs:
+        c.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK if selector == "chunk" else binding.SELECTOR_TOPK)
+    idx = torch.empty(k, device=dev, dtype=torch.int32)
+    rows = torch.empty(n * k, device=dev, dtype=torch.float32)
+    val = torch.empty(k, device=dev, dtype=torch.float32)
+    try:
+        for t in range(2 * n + 1):
+            g = workloads.gradients(w, t, dev, prof)
+            idx.fill_(-1); rows.fill_(float("nan")); val.fill_(float("nan"))
+            ctxs[t % n].select(g[t % n], mem[t % n], idx)
+            for i in range(n):
+                ctxs[i].compress(g[i], mem[i], idx, rows[i * k:(i + 1) * k])
+            for i in range(n):
+                if i % 2:                                  # fused and separate weight update must agree
+                    ctxs[i].reduce_rows(rows, val, idx, theta[i])
+                else:
+                    ctxs[i].reduce_rows(rows, val)
+                    ctxs[i].apply_update(theta[i], idx, val, lr)
+            torch.cuda.synchronize()
+            assert all(c.status() == binding.OK for c in ctxs)
+            idx_o, val_o, G_o = oracle.step([x.cpu().numpy() for x in g], m_o, th_o, t, k, beta, lr, selector=selector)
+            assert np.array_equal(idx.cpu().numpy(), idx_o)
+            assert np.array_equal(rows.cpu().numpy().reshape(n, k), G_o)
+            assert np.array_equal(val.cpu().numpy(), val_o)
+            for i in range(n):
+                assert np.array_equal(mem[i].cpu().numpy(), m_o[i])
+                assert np.array_equal(theta[i].cpu().numpy(), th_o)
+    finally:
+        for c in ctxs:
+            c.close()
+
+
+@pytest.mark.gpu
+def test_compress_rejects_a_malformed_index_list():
+    """An index list that is not strictly ascending, or reaches past d, sets the handle's status
+    instead of being applied out of bounds."""
+    import torch
+    from paper_2104_11125_b200 import binding
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    d, k = 10_000, 100
+    g = torch.randn(d, device=dev)
+    for bad in ("order", "range"):
+        m = torch.zeros(d, device=dev)
+        idx = torch.arange(0, 10 * k, 10, device=dev, dtype=torch.int32)
+        if bad == "order":
+            idx[7] = idx[6]
+        else:
+            idx[k - 1] = d
+        out = torch.empty(k, device=dev)
+        with sc.Context(d, 1, k, 0.1, 0.01) as ctx:
+            ctx.compress(g, m, idx, out)
+            torch.cuda.synchronize()
+            assert ctx.status() == binding.ERR_INTERNAL
+            with pytest.raises(sc.ScaleComError):
+                ctx.compress(g, m, idx, out)            # poisoned until reset
+            ctx.reset()
+            good = torch.arange(0, 10 * k, 10, device=dev, dtype=torch.int32)
+            ctx.compress(g, m, good, out)
+            torch.cuda.synchronize()
+            assert ctx.status() == binding.OK
+
+
+@pytest.mark.gpu
+def test_compress_takes_whatever_list_comes_next():
+    """The handle's bitmap is reused between calls: a list that differs from the one before it, or from what
+    a selection on the same handle left behind, must be applied alone."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2104_11125_b200 import binding
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    d, k, beta = 70_001, 700, 0.1
+    gen = torch.Generator(device=dev).manual_seed(5)
+    rng = np.random.default_rng(11)
+    m = torch.randn(d, device=dev, generator=gen)
+    m_o = m.cpu().numpy().copy()
+    out = torch.empty(k, device=dev)
+    own_idx = torch.empty(k, device=dev, dtype=torch.int32)
+    with sc.Context(d, 1, k, beta, 0.01) as ctx:
+        for it in range(6):
+            g = torch.randn(d, device=dev, generator=gen)
+            if it in (2, 4):                       # a selection writes its own set into the bitmap first
+                ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK if it == 4 else binding.SELECTOR_TOPK)
+                ctx.select(g, m, own_idx)
+            idx_o = np.sort(rng.choice(d, size=k, replace=False)).astype(np.int32)
+            if it == 5:
+                idx_o = np.arange(d - k, d, dtype=np.int32)     # a dense run up to the last coordinate
+            sel = np.zeros(d, np.uint8)
+            sel[idx_o] = 1
+            ctx.compress(g, m, torch.from_numpy(idx_o).to(dev), out)
+            torch.cuda.synchronize()
+            assert ctx.status() == binding.OK
+            gathered_o = oracle.learner(g.cpu().numpy(), m_o, idx_o, sel, beta)
+            assert np.array_equal(out.cpu().numpy(), gathered_o), it
+            assert np.array_equal(m.cpu().numpy(), m_o), it
