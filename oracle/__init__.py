@@ -63,6 +63,8 @@ def _load():
             f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, ctypes.c_int, vp, vp, vp]
             f = getattr(_lib, "oracle_layer_chunk_select_" + sfx); f.restype = ctypes.c_int
             f.argtypes = [vp, i32, vp, vp, vp, vp]
+            f = getattr(_lib, "oracle_layer_topk_" + sfx); f.restype = ctypes.c_int
+            f.argtypes = [vp, i32, vp, vp, vp, vp]
             f = getattr(_lib, "oracle_step_layers_" + sfx); f.restype = ctypes.c_int
             f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, ctypes.c_int, i32, vp, vp, vp, vp, vp]
             f = getattr(_lib, "oracle_mean_acc_" + sfx); f.restype = None; f.argtypes = [vp, vp, i32, i64, vp]
@@ -141,6 +143,20 @@ def layer_chunk_select(x: np.ndarray, sizes, keep):
     idx = np.empty(int(kp.sum()), np.int32)
     sel = np.empty(x.size, np.uint8)
     getattr(lib, "oracle_layer_chunk_select_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), sz.size, _p(sz), _p(kp), _p(idx), _p(sel))
+    return idx, sel
+
+
+def layer_topk(x: np.ndarray, sizes, keep):
+    """Exact top-k inside every layer (Eq. 2 applied per layer with Section 4's per-layer rates): layer s has
+    sizes[s] coordinates and keeps keep[s]; returns (idx int32[sum keep] ascending, sel uint8[d])."""
+    lib = _load()
+    sz = np.ascontiguousarray(sizes, np.int64)
+    kp = np.ascontiguousarray(keep, np.int64)
+    assert sz.size == kp.size and sz.sum() == x.size and np.all(kp >= 1) and np.all(kp <= sz)
+    idx = np.empty(int(kp.sum()), np.int32)
+    sel = np.empty(x.size, np.uint8)
+    if getattr(lib, "oracle_layer_topk_" + _sfx(x.dtype))(_p(_chk(x, x.dtype)), sz.size, _p(sz), _p(kp), _p(idx), _p(sel)) != 0:
+        raise MemoryError("oracle_layer_topk")
     return idx, sel
 
 
@@ -231,7 +247,7 @@ def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: boo
     if layers is not None:
         sz = np.ascontiguousarray(layers[0], np.int64)
         kp = np.ascontiguousarray(layers[1], np.int64)
-        assert selector == "chunk" and sz.sum() == d and kp.sum() == k and sz.size == kp.size
+        assert sz.sum() == d and kp.sum() == k and sz.size == kp.size
         nl, szp, kpp = sz.size, _p(sz), _p(kp)
     else:
         nl, szp, kpp = 0, None, None

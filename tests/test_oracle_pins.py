@@ -421,3 +421,43 @@ def test_layer_chunk_select():
     idx2, val, G = oracle.step(g, [a.copy() for a in m], None, 4, sum(keep), 0.5, 0.0, selector="chunk", layers=(sizes, keep))
     assert np.array_equal(idx2, oracle.layer_chunk_select(acc[4 % 3].copy(), sizes, keep)[0])
     np.testing.assert_allclose(val, acc[:, idx2].mean(axis=0), rtol=1e-13)
+
+
+# ---- exact top-k with per-layer rates (Eq. 2 inside each layer, Section 4's rates) -----------------
+def test_layer_topk():
+    sizes = [7, 64, 1, 300, 128, 40]
+    keep = [7, 2, 1, 3, 16, 5]                 # uncompressed layer, 32X, a single coordinate, 100X, 8X, 8X over ties
+    d = sum(sizes)
+    x = RNG.standard_normal(d).astype(np.float32)
+    x[80:90] = 0.0                              # zeros inside a layer (never picked while larger values remain)
+    x[500:540] = -0.25                          # the last layer is one 40-way tie: its 5 lowest indices win
+    x[510] = 0.25                               # the sign does not break the tie
+    idx, sel = oracle.layer_topk(x, sizes, keep)
+    assert idx.size == sum(keep) and np.all(np.diff(idx) > 0) and sel.sum() == sum(keep)
+    assert np.array_equal(np.flatnonzero(sel), idx)
+    key = key32(x).astype(np.int64)
+    off, expect = 0, []
+    for sz, kp in zip(sizes, keep):             # brute force by counting: p is kept iff fewer than keep precede it
+        for p in range(off, off + sz):
+            before = sum(1 for q in range(off, off + sz) if key[q] > key[p] or (key[q] == key[p] and q < p))
+            if before < kp:
+                expect.append(p)
+        off += sz
+    assert idx.tolist() == expect
+    assert idx[:7].tolist() == list(range(7))                          # keep = size: the layer is sent whole
+    assert idx[-5:].tolist() == [500, 501, 502, 503, 504]              # ties go to the lower index
+    # one layer is Eq. 2 on the whole vector
+    assert np.array_equal(oracle.layer_topk(x, [d], [13])[0], oracle.topk(x, 13)[0])
+    # moving a layer boundary changes the result (the layers are searched separately)
+    y = np.arange(1, 21, dtype=np.float32)
+    assert oracle.layer_topk(y, [10, 10], [1, 1])[0].tolist() == [9, 19]
+    assert oracle.layer_topk(y, [15, 5], [1, 1])[0].tolist() == [14, 19]
+    assert oracle.topk(y, 2)[0].tolist() == [18, 19]
+    # the step with layers and the exact selector is the same algorithm with that index set
+    g = [RNG.standard_normal(d) for _ in range(3)]
+    m = [RNG.standard_normal(d) for _ in range(3)]
+    acc = np.stack([a + b for a, b in zip(m, g)])
+    idx2, val, G = oracle.step(g, [a.copy() for a in m], None, 4, sum(keep), 0.5, 0.0, selector="topk", layers=(sizes, keep))
+    assert np.array_equal(idx2, oracle.layer_topk(acc[4 % 3].copy(), sizes, keep)[0])
+    np.testing.assert_allclose(val, acc[:, idx2].mean(axis=0), rtol=1e-13)
+    assert np.array_equal(G, acc[:, idx2])
