@@ -128,7 +128,8 @@ int scalecom_set_gathered(scalecom_ctx* ctx, float* dev_gathered);
  * keep[s] of them by the chunk-wise rule applied inside the layer (keep[s] == sizes[s]: sent whole).
  *   nlayers  1 .. 2048, or 0 to go back to one rate for the whole vector.
  *   sizes, keep  HOST int64[nlayers]; sizes[s] >= 1, 1 <= keep[s] <= sizes[s], sum sizes = d, sum keep = k.
- * Only SCALECOM_SELECTOR_CHUNK looks at the layers; the exact top-k selector ignores them.
+ * SCALECOM_SELECTOR_CHUNK and SCALECOM_SELECTOR_LAYER_TOPK look at the layers; SCALECOM_SELECTOR_TOPK
+ * (Eq. 2 over the whole vector) ignores them.
  * Waits for the stream.  Errors: NULL_PTR, INVALID_ARG, ALLOC, CUDA.
  */
 int scalecom_set_layers(scalecom_ctx* ctx, int32_t nlayers, const int64_t* sizes, const int64_t* keep);
@@ -197,19 +198,25 @@ int scalecom_reset(scalecom_ctx* ctx);
                                             Appendix E -- the d coordinates form k consecutive chunks,
                                             chunk j = [floor(j*d/k), floor((j+1)*d/k)), and each keeps its
                                             largest-magnitude coordinate (lower index on ties).  Steps 1, 3,
-                                            4, 5 are unchanged.  First use allocates 8*k bytes             */
+                                            4, 5 are unchanged.  First use allocates 8*k bytes;
+                                            SCALECOM_SELECTOR_LAYER_TOPK: Eq. 2 applied inside every layer
+                                            set by scalecom_set_layers -- layer s keeps its keep[s] largest
+                                            magnitudes, ties to the lower index (steps and scalecom_select
+                                            return BAD_STATE while no layers are set).  Its first launch
+                                            after scalecom_set_layers allocates 8 KB per layer             */
 #define SCALECOM_OPT_KERNEL_SPANS     7  /* 1: every kernel of a step records the time from its first block's
                                             start to its last block's end on the GPU's nanosecond timer
                                             (two atomics per block); read with scalecom_kernel_span_ms     */
 #define SCALECOM_SELECTOR_TOPK  0
 #define SCALECOM_SELECTOR_CHUNK 1
+#define SCALECOM_SELECTOR_LAYER_TOPK 2
 int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 
 /* Items for scalecom_query (each synchronises the stream when it reads device state). */
 #define SCALECOM_Q_WORKSPACE_BYTES  1  /* device bytes owned by the handle                                    */
 #define SCALECOM_Q_LAST_TOPK_PATH   2  /* last step's selection path: 0 = sampled pre-filter, 1 = full select,
                                           2 = pre-filter started from the previous step's threshold,
-                                          3 = chunk-wise selector                                             */
+                                          3 = chunk-wise selector, 4 = exact top-k per layer                  */
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */

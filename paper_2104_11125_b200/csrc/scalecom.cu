@@ -12,6 +12,7 @@
 #include "chunk_select.cuh"
 #include "diagnostics.cuh"
 #include "exchange.cuh"
+#include "layer_topk.cuh"
 #include "learner_pass.cuh"
 #include "topk_select.cuh"
 
@@ -47,6 +48,9 @@ struct scalecom_ctx {
     int selector = SCALECOM_SELECTOR_TOPK;
     unsigned long long* chunk_best = nullptr;   // [k], allocated when the chunk-wise selector is first chosen
     uint32_t chunk_blocks = 0;
+    void* lt_ws = nullptr;             // scratch of the per-layer exact selector (sized by nlayers), or nullptr
+    size_t lt_bytes = 0;
+    uint32_t lt_blocks = 0;
     uint32_t nlayers = 0;              // per-layer rates of the chunk-wise selector (0: one rate for the whole vector)
     uint32_t* layer_tab = nullptr;     // device [2][nlayers + 1]: coordinate offsets, chunk offsets
     uint32_t* one_layer_tab = nullptr; // device {0, d, 0, k}: the whole vector as one layer
@@ -116,6 +120,56 @@ cudaError_t launch_chunk(const scalecom_ctx* c, const ChunkParams& P) {
     return cudaLaunchCooperativeKernel(fn, dim3(c->chunk_blocks), dim3(CS_THREADS), args, 0, c->stream);
 }
 
+// Scratch of the per-layer exact selector, made at the first launch after the layers were set.
+int ensure_layer_ws(scalecom_ctx* c) {
+    if (c->lt_ws) return SCALECOM_OK;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, layer_topk_kernel<true>, LT_THREADS, sizeof(LayerTopkShared)) !=
+            cudaSuccess || occ < 1)
+        return SCALECOM_ERR_CUDA;
+    if (occ > LT_BLOCKS_PER_SM) occ = LT_BLOCKS_PER_SM;
+    c->lt_blocks = uint32_t(c->sms * occ);
+    const size_t nl = c->nlayers;
+    c->lt_bytes = nl * LT_BINS * 4 + nl * 16 + 256 + size_t(c->lt_blocks) * 4;
+    if (cudaMalloc(&c->lt_ws, c->lt_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        c->lt_ws = nullptr;
+        return SCALECOM_ERR_ALLOC;
+    }
+    if (cudaMemsetAsync(c->lt_ws, 0, c->lt_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+    return SCALECOM_OK;
+}
+
+LayerTopkParams make_layer_params(const scalecom_ctx* c, const float* g, const float* m, int32_t* out_idx,
+                                  unsigned long long* span_slot) {
+    LayerTopkParams P;
+    const size_t nl = c->nlayers;
+    char* base = static_cast<char*>(c->lt_ws);
+    P.g = g; P.m = m; P.d = uint32_t(c->d); P.k = uint32_t(c->k);
+    P.spin_limit = c->spin_limit;
+    P.nl = c->nlayers;
+    P.layer_off = c->layer_tab;
+    P.layer_k0 = c->layer_tab + (nl + 1);
+    P.ghist = reinterpret_cast<uint32_t*>(base);
+    P.lstate = reinterpret_cast<uint4*>(base + nl * LT_BINS * 4);
+    P.tie_flag = reinterpret_cast<uint32_t*>(base + nl * LT_BINS * 4 + nl * 16);
+    P.block_tot = reinterpret_cast<uint32_t*>(base + nl * LT_BINS * 4 + nl * 16 + 256);
+    P.bitmap = c->bitmap; P.tile_prefix = c->tile_prefix; P.ntiles = c->ntiles;
+    P.ctrl = c->ctrl;
+    P.barrier = c->barrier + 16;               // its own arrival counter (its grid differs from the other selectors')
+    P.out_idx = out_idx;
+    P.spans = span_slot;
+    return P;
+}
+
+template <bool VEC>
+cudaError_t launch_layer_topk(const scalecom_ctx* c, const LayerTopkParams& P) {
+    c->bitmap_zero = false;
+    void* args[] = {const_cast<LayerTopkParams*>(&P)};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&layer_topk_kernel<VEC>), dim3(c->lt_blocks),
+                                       dim3(LT_THREADS), args, sizeof(LayerTopkShared), c->stream);
+}
+
 template <int N, bool VEC, int T, int L = LP_UNROLL / T, bool ONE = false>
 cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem, const LearnerParams& P) {
     PtrTable<N> tab;
@@ -158,6 +212,7 @@ int init_workspace(scalecom_ctx* c) {
     if (cudaMemsetAsync(c->ws, 0, c->ctrl_region_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     if (c->chunk_best && cudaMemsetAsync(c->chunk_best, 0, size_t(c->k) * 8, c->stream) != cudaSuccess)
         return SCALECOM_ERR_CUDA;
+    if (c->lt_ws && cudaMemsetAsync(c->lt_ws, 0, c->lt_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     return SCALECOM_OK;
 }
 
@@ -220,6 +275,11 @@ TopkParams make_topk_params(const scalecom_ctx* c, const float* g, const float* 
 int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float* weights, int64_t t, int32_t* out_idx,
             float* out_val) {
     const int leader = int(t % c->n);
+    if (c->selector == SCALECOM_SELECTOR_LAYER_TOPK) {
+        if (!c->nlayers) return SCALECOM_ERR_BAD_STATE;        // this selector has no meaning without layers
+        const int rc = ensure_layer_ws(c);
+        if (rc != SCALECOM_OK) return rc;
+    }
 
     unsigned long long* const span_slot =
         (c->span_timing && c->spans) ? c->spans + 4 * (c->span_steps % scalecom_ctx::EV_RING) : nullptr;
@@ -265,6 +325,9 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
         cp.layer_off = c->nlayers ? c->layer_tab : c->one_layer_tab;
         cp.layer_chunk0 = cp.layer_off + (cp.nl + 1);
         e = vec_leader ? launch_chunk<true>(c, cp) : launch_chunk<false>(c, cp);
+    } else if (c->selector == SCALECOM_SELECTOR_LAYER_TOPK) {
+        const LayerTopkParams P = make_layer_params(c, tp.g, tp.m, nullptr, span_slot);
+        e = vec_leader ? launch_layer_topk<true>(c, P) : launch_layer_topk<false>(c, P);
     } else {
         e = vec_leader ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
     }
@@ -469,6 +532,7 @@ void scalecom_destroy(scalecom_ctx* c) {
     }
     cudaFree(c->ws);
     cudaFree(c->chunk_best);
+    cudaFree(c->lt_ws);
     cudaFree(c->layer_tab);
     cudaFree(c->one_layer_tab);
     cudaFree(c->spans);
@@ -499,7 +563,9 @@ int scalecom_set_layers(scalecom_ctx* c, int32_t nlayers, const int64_t* sizes, 
     if (cudaStreamSynchronize(c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;   // a step may still read the old table
     if (nlayers == 0) {
         cudaFree(c->layer_tab);
+        cudaFree(c->lt_ws);
         c->layer_tab = nullptr;
+        c->lt_ws = nullptr;
         c->nlayers = 0;
         return SCALECOM_OK;
     }
@@ -531,6 +597,8 @@ int scalecom_set_layers(scalecom_ctx* c, int32_t nlayers, const int64_t* sizes, 
             rc = SCALECOM_ERR_CUDA;
         } else {
             cudaFree(c->layer_tab);
+            cudaFree(c->lt_ws);                    // sized by the number of layers: made again at the next launch
+            c->lt_ws = nullptr;
             c->layer_tab = dev;
             c->nlayers = uint32_t(nlayers);
         }
@@ -579,6 +647,12 @@ int scalecom_select(scalecom_ctx* c, const float* g, const float* m, int32_t* ou
         cp.layer_off = c->nlayers ? c->layer_tab : c->one_layer_tab;
         cp.layer_chunk0 = cp.layer_off + (cp.nl + 1);
         e = vec ? launch_chunk<true>(c, cp) : launch_chunk<false>(c, cp);
+    } else if (c->selector == SCALECOM_SELECTOR_LAYER_TOPK) {
+        if (!c->nlayers) return SCALECOM_ERR_BAD_STATE;
+        const int rc = ensure_layer_ws(c);
+        if (rc != SCALECOM_OK) return rc;
+        const LayerTopkParams P = make_layer_params(c, g, m, out_idx, nullptr);
+        e = vec ? launch_layer_topk<true>(c, P) : launch_layer_topk<false>(c, P);
     } else {
         // one vector, one hint slot: the handle of a learner-per-GPU rank always sees the same learner
         TopkParams tp = make_topk_params(c, g, m, c->leader_hint, true, nullptr);
@@ -709,7 +783,8 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
             return SCALECOM_OK;
         }
         case SCALECOM_OPT_SELECTOR: {
-            if (value != SCALECOM_SELECTOR_TOPK && value != SCALECOM_SELECTOR_CHUNK) return SCALECOM_ERR_INVALID_ARG;
+            if (value != SCALECOM_SELECTOR_TOPK && value != SCALECOM_SELECTOR_CHUNK && value != SCALECOM_SELECTOR_LAYER_TOPK)
+                return SCALECOM_ERR_INVALID_ARG;
             if (value == SCALECOM_SELECTOR_CHUNK && !c->chunk_best) {
                 DeviceGuard guard(c->device);
                 int occ = 0;

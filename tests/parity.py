@@ -71,7 +71,8 @@ def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exac
         ctx.set_option(binding.OPT_FORCE_EXACT_PATH, int(force_exact))
         ctx.set_option(binding.OPT_FUSE_UPDATE, int(fuse_update))
         ctx.set_option(binding.OPT_USE_HINT, int(use_hint))
-        ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK if selector == "chunk" else binding.SELECTOR_TOPK)
+        ctx.set_option(binding.OPT_SELECTOR, {"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
+                                              "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
         if layers is not None:
             ctx.set_layers(*layers)
         for s, grads in enumerate(grads_per_step):
@@ -82,7 +83,10 @@ def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exac
             assert ctx.status() == 0, "%s step %d: device status %d" % (tag, s, ctx.status())
             paths.append(ctx.query(binding.Q_LAST_TOPK_PATH))
             g_np = [g.cpu().numpy() for g in grads]
-            idx_o, val_o, G_o = oracle.step(g_np, m_o, th_o, t, k, beta, lr, selector=selector, layers=layers)
+            # "layer_topk" is the oracle's exact selector applied inside the layers
+            idx_o, val_o, G_o = oracle.step(g_np, m_o, th_o, t, k, beta, lr,
+                                            selector="topk" if selector == "layer_topk" else selector,
+                                            layers=layers if selector != "topk" else None)
             assert_step_matches("%s step %d" % (tag, s), idx.cpu().numpy(), val.cpu().numpy(),
                                 G.cpu().numpy().reshape(n, k), [x.cpu().numpy() for x in m_g],
                                 th_g.cpu().numpy() if th_g is not None else None,

@@ -421,3 +421,81 @@ def test_layer_rates_resnet50_rule():
     w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
     paths = _parity().workload_case(w2, 3, DEV, selector="chunk", layers=(sizes, keep))
     assert all(x == 3 for x in paths)
+
+
+# ---- exact top-k inside every layer (Eq. 2 per layer with Section 4's per-layer rates) --------------------
+def test_layer_topk_small_cases():
+    rng = np.random.default_rng(37)
+    p = _parity()
+    for sizes, keep in [([7, 64, 1, 300, 128], [7, 2, 1, 3, 16]),
+                        ([5000], [50]),
+                        ([1] * 40, [1] * 40),
+                        ([1000, 3000, 2000, 4099], [1000, 30, 5, 4099]),
+                        ([2048, 2048, 4096, 100_000, 64, 64, 3], [20, 2048, 1, 1000, 64, 1, 2]),
+                        ([300_000, 17, 200_001], [3000, 17, 20])]:
+        d, k = sum(sizes), sum(keep)
+        g = [_t(rng.standard_normal(d)) for _ in range(3)]
+        m0 = [torch.zeros(d, device=DEV) for _ in range(3)]
+        for offset in (0, 1):
+            paths = p.run_and_compare([g] * 3, m0, torch.linspace(-1, 1, d, device=DEV), k, 0.5, 0.25, offset=offset,
+                                      selector="layer_topk", layers=(sizes, keep), tag="layer top-k %d" % len(sizes))
+            assert all(x == binding_path_layer() for x in paths)
+
+
+def binding_path_layer():
+    from paper_2104_11125_b200 import binding
+    return binding.PATH_LAYER_TOPK
+
+
+def test_layer_topk_ties_across_the_boundary():
+    """Layers whose k-th magnitude is shared by more coordinates than may be kept: the lowest indices win.
+    A constant layer, an all-zero layer, a layer of two values, next to an ordinary one."""
+    rng = np.random.default_rng(41)
+    sizes = [5000, 3000, 70_000, 4000, 1]
+    keep = [50, 3000 - 1, 700, 17, 1]
+    d, k = sum(sizes), sum(keep)
+    base = rng.standard_normal(d).astype(np.float32)
+    base[0:5000] = 0.5                                        # constant: 50 of 5000 equal keys
+    base[5000:8000] = 0.0                                     # all zero, all but one kept
+    base[8000:78_000] = np.where(rng.random(70_000) < 0.5, 1.0, -2.0).astype(np.float32)   # two magnitudes
+    g = [_t(base), _t(base * 2), _t(-base)]
+    m0 = [torch.zeros(d, device=DEV) for _ in range(3)]
+    p = _parity()
+    for offset in (0, 3):
+        paths = p.run_and_compare([g] * 3, m0, None, k, 0.5, 0.25, offset=offset, selector="layer_topk",
+                                  layers=(sizes, keep), tag="layer top-k ties")
+        assert all(x == binding_path_layer() for x in paths)
+
+
+def test_layer_topk_needs_layers():
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    d, k = 1000, 10
+    g = [torch.randn(d, device=DEV)]
+    m = [torch.zeros(d, device=DEV)]
+    idx = torch.empty(k, device=DEV, dtype=torch.int32)
+    val = torch.empty(k, device=DEV)
+    with sc.Context(d, 1, k, 0.5, 0.1) as ctx:
+        ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_LAYER_TOPK)
+        with pytest.raises(sc.ScaleComError) as ei:
+            ctx.step(g, m, None, 0, idx, val)
+        assert ei.value.code == binding.ERR_BAD_STATE
+        ctx.set_layers([400, 600], [4, 6])
+        ctx.step(g, m, None, 0, idx, val)
+        assert ctx.status() == 0
+        got = idx.cpu().numpy()
+        assert (got[:4] < 400).all() and (got[4:] >= 400).all()
+        ctx.set_layers([1000], [10])                          # one layer: Eq. 2 on the whole vector
+        m2 = [torch.zeros(d, device=DEV)]
+        ctx.step(g, m2, None, 0, idx, val)
+        want = np.sort(np.argsort(-np.abs(g[0].cpu().numpy()), kind="stable")[:k])
+        assert np.array_equal(idx.cpu().numpy(), want)
+
+
+def test_layer_topk_resnet50_rule():
+    """The paper's per-layer rates on the ResNet-50-shaped workload at a test size, exact selection per tensor."""
+    w = W.RESNET50.scaled(2_000_003)
+    sizes, keep = W.resnet50_layer_keep(w)
+    w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
+    paths = _parity().workload_case(w2, 3, DEV, selector="layer_topk", layers=(sizes, keep))
+    assert all(x == binding_path_layer() for x in paths)
