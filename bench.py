@@ -44,8 +44,9 @@ def parse_args():
     ap.add_argument("--batches", type=int, default=MAX_BATCHES,
                     help="distinct gradient batches kept in HBM (steps cycle through them); small values keep "
                          "the footprint low for profiler captures")
-    ap.add_argument("--selector", default="topk", choices=["topk", "chunk"],
-                    help="leader selection: exact top-k (the headline path) or the chunk-wise selector")
+    ap.add_argument("--selector", default="topk", choices=["topk", "chunk", "layer_topk"],
+                    help="leader selection: exact top-k (the headline path), the chunk-wise selector, or exact top-k "
+                         "inside every layer (needs --layers)")
     ap.add_argument("--layers", action="store_true",
                     help="with --selector chunk on a ResNet-50-shaped workload: the paper's per-layer rate rule "
                          "(25X / 50X / 400X, first layer whole) instead of one rate; k becomes the sum of the layers' keeps")
@@ -163,15 +164,16 @@ def run_reference(args):
     prof = W.profile(w, "cpu")
     nb = min(args.steps + args.warmup, 4)
     batches = [[g.numpy() for g in W.gradients(w, s, "cpu", prof)] for s in range(nb)]
+    osel = "chunk" if args.selector == "chunk" else "topk"        # (per-layer rates are not part of this arm)
     m = [x.numpy() for x in W.initial_memory(w, "cpu")]
     th = W.initial_weights(w, "cpu").numpy()
     t = 0
     for _ in range(args.warmup):
-        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False, selector=args.selector)
+        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False, selector=osel)
         t += 1
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False, selector=args.selector)
+        oracle.step(batches[t % nb], m, th, t, w.k, w.beta, w.lr, want_gathered=False, selector=osel)
         t += 1
     dt = time.perf_counter() - t0
     value = w.n * w.d * args.steps / dt
@@ -198,7 +200,8 @@ def time_oracle(w, batches_dev, steps=2, selector="topk", layers=None):
     for s in range(steps):
         g = [x.cpu().numpy() for x in batches_dev[s % len(batches_dev)]]
         t0 = time.perf_counter()
-        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False, selector=selector, layers=layers)
+        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False,
+                    selector="topk" if selector == "layer_topk" else selector, layers=layers)
         dt += time.perf_counter() - t0
     return {"value": w.n * w.d * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
             "sample": "%d full steps of the bench workload (n=%d, d=%d, k=%d), %.1f s" % (steps, w.n, w.d, w.k, dt)}
@@ -334,8 +337,8 @@ def main():
     w = get_workload(args.workload)
     layers = None
     if args.layers:
-        if args.selector != "chunk" or w.kind != "resnet50":
-            raise SystemExit("--layers needs --selector chunk and a ResNet-50-shaped workload")
+        if args.selector == "topk" or w.kind != "resnet50":
+            raise SystemExit("--layers needs --selector chunk or layer_topk and a ResNet-50-shaped workload")
         layers = W.resnet50_layer_keep(w)
         w = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(layers[1]), w.beta, w.lr, w.steps, w.c)
     K, Wm = args.steps, max(args.warmup, 3)
@@ -349,6 +352,10 @@ def main():
 
     stream = torch.cuda.Stream(device=dev)
     ctx = sc.Context(w.d, w.n, w.k, w.beta, w.lr, stream=stream)
+    if args.selector == "layer_topk":
+        if layers is None:
+            raise SystemExit("--selector layer_topk needs --layers")
+        ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_LAYER_TOPK)
     if args.selector == "chunk":
         ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK)
     if layers is not None:

@@ -21,11 +21,22 @@
 
 namespace sc {
 
+#ifndef SC_LT_BLOCKS_PER_SM
+#define SC_LT_BLOCKS_PER_SM 2
+#endif
+#ifndef SC_LT_UNROLL
+#define SC_LT_UNROLL 2
+#endif
+
 constexpr int LT_THREADS = 512;
-constexpr int LT_BLOCKS_PER_SM = 2;
+constexpr int LT_BLOCKS_PER_SM = SC_LT_BLOCKS_PER_SM;
+constexpr int LT_UNROLL = SC_LT_UNROLL;             // spans whose loads a thread has in flight
 constexpr uint32_t LT_SPAN = LT_THREADS * 4;        // coordinates a block takes per iteration (two tiles)
 constexpr uint32_t LT_BINS = 2048;                  // widest digit: 11 bits
 constexpr uint32_t LT_NOSPLIT = 0xFFFFFFFFu;
+// Words between two layers' rows of the global histogram: an odd number of 128-byte lines, so that the same
+// bin of different layers does not sit a power of two apart.
+constexpr uint32_t LT_ROW = LT_BINS + 32;
 
 struct LayerTopkParams {
     const float* g;
@@ -35,7 +46,7 @@ struct LayerTopkParams {
     uint32_t nl;
     const uint32_t* layer_off;          // [nl + 1] first coordinate of each layer
     const uint32_t* layer_k0;           // [nl + 1] prefix sums of keep[]
-    uint32_t* ghist;                    // [nl * LT_BINS], zero on entry, left zero
+    uint32_t* ghist;                    // [nl * LT_ROW], zero on entry, left zero
     uint4* lstate;                      // [nl] {prefix or T, still to keep, split flag, offset prefix or last kept offset}
     uint32_t* tie_flag;                 // one word, zero on entry, left zero
     uint32_t* block_tot;                // [grid]
@@ -126,11 +137,39 @@ __device__ __forceinline__ void lt_flush(LayerTopkShared& S, uint32_t* ghist, ui
     for (uint32_t i = threadIdx.x; i < LT_BINS; i += LT_THREADS) {
         const uint32_t v = S.hist[i];
         if (v) {
-            atomicAdd(&ghist[size_t(layer) * LT_BINS + i], v);
+            atomicAdd(&ghist[size_t(layer) * LT_ROW + i], v);
             S.hist[i] = 0;
         }
     }
     __syncthreads();
+}
+
+// This thread's quads of spans sp0 .. sp0 + LT_UNROLL - 1 (those below span_hi and d).  When all of them are
+// whole the loads carry no predicate, which is what keeps all of them in flight at once.
+template <bool VEC>
+__device__ __forceinline__ void lt_load_spans(const LayerTopkParams& P, uint32_t sp0, uint32_t span_hi,
+                                              float (&gv)[LT_UNROLL][4], float (&mv)[LT_UNROLL][4]) {
+    const uint32_t tid = threadIdx.x, d = P.d;
+    const bool whole = VEC && sp0 + LT_UNROLL <= span_hi && uint64_t(sp0 + LT_UNROLL) * LT_SPAN <= d;   // uniform
+    if (whole) {
+#pragma unroll
+        for (int u = 0; u < LT_UNROLL; ++u) {
+            const uint32_t p = (sp0 + u) * LT_SPAN + tid * 4u;
+            const float4 a = *reinterpret_cast<const float4*>(P.g + p);
+            const float4 b = *reinterpret_cast<const float4*>(P.m + p);
+            gv[u][0] = a.x; gv[u][1] = a.y; gv[u][2] = a.z; gv[u][3] = a.w;
+            mv[u][0] = b.x; mv[u][1] = b.y; mv[u][2] = b.z; mv[u][3] = b.w;
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < LT_UNROLL; ++u) {
+            const uint32_t p = (sp0 + u) * LT_SPAN + tid * 4u;
+            if (sp0 + u < span_hi && p < d) {
+                load_quad_stream<VEC>(P.g, p, d, gv[u]);
+                load_quad_stream<VEC>(P.m, p, d, mv[u]);
+            }
+        }
+    }
 }
 
 // One counting pass over this block's spans [span_lo, span_hi).
@@ -141,32 +180,56 @@ __device__ __forceinline__ void lt_stream_pass(const LayerTopkParams& P, LayerTo
     uint32_t cur = layer_first;                 // layer of this thread's quad (moves forward only)
     uint32_t cf = layer_first, cl = layer_first;        // layers of the span's first and last coordinate (uniform)
     uint32_t hist_layer = LT_NOSPLIT;           // layer whose counts the shared histogram holds (uniform)
-    for (uint32_t sp = span_lo; sp < span_hi; ++sp) {
-        const uint32_t p0 = sp * LT_SPAN, pe = min(p0 + LT_SPAN, d) - 1u;
-        while (p0 >= S.off[cf + 1]) ++cf;
-        while (pe >= S.off[cl + 1]) ++cl;
-        const bool uniform = cf == cl;
-        if (uniform && hist_layer != cf) {
-            if (hist_layer != LT_NOSPLIT) lt_flush(S, P.ghist, hist_layer);
-            hist_layer = cf;
+    constexpr int U = PS < 3 ? LT_UNROLL : 1;   // the tie rounds read only the spans of layers with a tie to split
+    for (uint32_t sp0 = span_lo; sp0 < span_hi; sp0 += U) {
+        if (PS >= 3) {
+            const uint32_t p0 = sp0 * LT_SPAN, pe = min(p0 + LT_SPAN, d) - 1u;
+            while (p0 >= S.off[cf + 1]) ++cf;
+            while (pe >= S.off[cl + 1]) ++cl;
+            bool any = false;
+            for (uint32_t s = cf; s <= cl; ++s) any = any || S.w[s] != LT_NOSPLIT;
+            if (!any) continue;                                             // uniform
         }
-        const uint32_t p = p0 + tid * 4u;
-        if (p >= d) continue;                   // (uniform-layer decisions above are already taken)
-        float gv[4], mv[4];
-        load_quad_stream<VEC>(P.g, p, d, gv);
-        load_quad_stream<VEC>(P.m, p, d, mv);
-        while (p >= S.off[cur + 1]) ++cur;
-        uint32_t s = cur;
+        // all loads of U spans first, then the counting (which may stop for a flush in between)
+        float gv[LT_UNROLL][4], mv[LT_UNROLL][4];
+        if (PS < 3) {
+            lt_load_spans<VEC>(P, sp0, span_hi, gv, mv);
+        } else {
+            const uint32_t p = sp0 * LT_SPAN + tid * 4u;
+            if (p < d) {
+                load_quad_stream<VEC>(P.g, p, d, gv[0]);
+                load_quad_stream<VEC>(P.m, p, d, mv[0]);
+            }
+        }
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint32_t pc = p + c;
-            if (pc >= d) break;
-            while (pc >= S.off[s + 1]) ++s;
-            const uint32_t key = mag_key(__fadd_rn(mv[c], gv[c]));
-            uint32_t dg;
-            if (lt_match<PS>(key, pc - S.off[s], S.x[s], S.w[s], &dg)) {
-                if (uniform) atomicAdd(&S.hist[dg], 1u);
-                else atomicAdd(&P.ghist[size_t(s) * LT_BINS + dg], 1u);
+        for (int u = 0; u < U; ++u) {
+            const uint32_t sp = sp0 + u;
+            if (sp >= span_hi) break;                                       // uniform
+            const uint32_t p0 = sp * LT_SPAN, pe = min(p0 + LT_SPAN, d) - 1u;
+            while (p0 >= S.off[cf + 1]) ++cf;
+            while (pe >= S.off[cl + 1]) ++cl;
+            const bool uniform = cf == cl;
+            if (uniform && hist_layer != cf) {
+                if (hist_layer != LT_NOSPLIT) lt_flush(S, P.ghist, hist_layer);
+                hist_layer = cf;
+            }
+            const uint32_t p = p0 + tid * 4u;
+            if (p >= d) continue;               // (the uniform decisions above are already taken)
+            while (p >= S.off[cur + 1]) ++cur;
+            uint32_t s = cur;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t pc = p + c;
+                if (pc >= d) break;
+                while (pc >= S.off[s + 1]) ++s;
+                const uint32_t key = mag_key(__fadd_rn(mv[u][c], gv[u][c]));
+                uint32_t dg;
+                if (lt_match<PS>(key, pc - S.off[s], S.x[s], S.w[s], &dg)) {
+                    // a span where layers meet counts straight into their global rows (taking such a span through
+                    // the shared histogram one layer at a time measured 20 % slower per pass)
+                    if (uniform) atomicAdd(&S.hist[dg], 1u);
+                    else atomicAdd(&P.ghist[size_t(s) * LT_ROW + dg], 1u);
+                }
             }
         }
     }
@@ -182,11 +245,9 @@ __device__ __forceinline__ void lt_find_round(const LayerTopkParams& P, LayerTop
         uint4 st = make_uint4(0, 0, 0, LT_NOSPLIT);
         if (PS > 0) st = __ldcg(&P.lstate[s]);
         if (PS >= 3 && st.z == 0) continue;                                // uniform: no tie to split in this layer
-        for (uint32_t i = tid; i < LT_BINS; i += LT_THREADS) {
-            uint32_t* row = &P.ghist[size_t(s) * LT_BINS + i];
-            S.hist[i] = __ldcg(row);
-            *row = 0;
-        }
+        // (an exchange, not a load and a store: one trip to L2 per word)
+        for (uint32_t i = tid; i < LT_BINS; i += LT_THREADS)
+            S.hist[i] = atomicExch(&P.ghist[size_t(s) * LT_ROW + i], 0u);
         __syncthreads();
         const uint32_t r = PS == 0 ? P.layer_k0[s + 1] - P.layer_k0[s] : st.y;
         lt_block_find<(PS < 3)>(S, nbins, r);
@@ -246,22 +307,34 @@ __global__ void __launch_bounds__(LT_THREADS, LT_BLOCKS_PER_SM) layer_topk_kerne
     for (size_t i = size_t(blockIdx.x) * LT_THREADS + tid; i <= P.ntiles; i += size_t(nblocks) * LT_THREADS)
         P.tile_prefix[i] = 0;
 
+    // phase time stamps of block 0 (low word of the nanosecond global timer), for profiling only
+#define LT_STAMP(i) do { if (blockIdx.x == 0 && tid == 0) { uint32_t ts_; asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(ts_)); \
+                                                            P.ctrl[8 + (i)] = ts_; } } while (0)
+    LT_STAMP(0);
     // ---------------- three rounds over the magnitude key ---------------------------------------------
     lt_stream_pass<0, VEC>(P, S, span_lo, span_hi, lf);
+    LT_STAMP(1);
     if (!grid_barrier(gb, &S.flag)) return;
+    LT_STAMP(2);
     lt_find_round<0>(P, S);
+    LT_STAMP(3);
     if (!grid_barrier(gb, &S.flag)) return;
     if (have) lt_load_state(P, S, lf, ll);
+    LT_STAMP(4);
     lt_stream_pass<1, VEC>(P, S, span_lo, span_hi, lf);
+    LT_STAMP(5);
     if (!grid_barrier(gb, &S.flag)) return;
     lt_find_round<1>(P, S);
     if (!grid_barrier(gb, &S.flag)) return;
     if (have) lt_load_state(P, S, lf, ll);
+    LT_STAMP(6);
     lt_stream_pass<2, VEC>(P, S, span_lo, span_hi, lf);
+    LT_STAMP(7);
     if (!grid_barrier(gb, &S.flag)) return;
     lt_find_round<2>(P, S);
     if (!grid_barrier(gb, &S.flag)) return;
     if (have) lt_load_state(P, S, lf, ll);
+    LT_STAMP(8);
 
     // ---------------- ties across a layer's boundary: three rounds over the offset ---------------------
     if (__ldcg(P.tie_flag) != 0u) {                                          // the same answer in every block
@@ -286,36 +359,40 @@ __global__ void __launch_bounds__(LT_THREADS, LT_BLOCKS_PER_SM) layer_topk_kerne
     uint32_t mine = 0;                                                       // coordinates this thread selected
     {
         uint32_t cur = lf;
-        for (uint32_t sp = span_lo; sp < span_hi; ++sp) {
-            const uint32_t p = sp * LT_SPAN + tid * 4u;
-            uint32_t nib = 0;
-            if (p < d) {
-                float gv[4], mv[4];
-                load_quad_stream<VEC>(P.g, p, d, gv);
-                load_quad_stream<VEC>(P.m, p, d, mv);
-                while (p >= S.off[cur + 1]) ++cur;
-                uint32_t s = cur;
+        for (uint32_t sp0 = span_lo; sp0 < span_hi; sp0 += LT_UNROLL) {
+            float gv[LT_UNROLL][4], mv[LT_UNROLL][4];
+            lt_load_spans<VEC>(P, sp0, span_hi, gv, mv);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t pc = p + c;
-                    if (pc >= d) break;
-                    while (pc >= S.off[s + 1]) ++s;
-                    const uint32_t key = mag_key(__fadd_rn(mv[c], gv[c]));
-                    const uint32_t T = S.x[s], w = S.w[s];
-                    if (key > T || (key == T && (w == LT_NOSPLIT || pc - S.off[s] <= w))) nib |= 1u << c;
+            for (int u = 0; u < LT_UNROLL; ++u) {
+                const uint32_t sp = sp0 + u;
+                if (sp >= span_hi) break;                                    // uniform
+                const uint32_t p = sp * LT_SPAN + tid * 4u;
+                uint32_t nib = 0;
+                if (p < d) {
+                    while (p >= S.off[cur + 1]) ++cur;
+                    uint32_t s = cur;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t pc = p + c;
+                        if (pc >= d) break;
+                        while (pc >= S.off[s + 1]) ++s;
+                        const uint32_t key = mag_key(__fadd_rn(mv[u][c], gv[u][c]));
+                        const uint32_t T = S.x[s], w = S.w[s];
+                        if (key > T || (key == T && (w == LT_NOSPLIT || pc - S.off[s] <= w))) nib |= 1u << c;
+                    }
                 }
+                // eight neighbouring threads make one bitmap word
+                uint32_t word = nib << ((lane & 7u) * 4u);
+                word |= __shfl_xor_sync(FULL, word, 1);
+                word |= __shfl_xor_sync(FULL, word, 2);
+                word |= __shfl_xor_sync(FULL, word, 4);
+                const uint32_t widx = sp * (LT_SPAN / 32u) + (tid >> 3);
+                if ((lane & 7u) == 0u && widx < P.ntiles * 32u) P.bitmap[widx] = word;
+                const uint32_t wcnt = warp_sum(__popc(nib));                 // a warp lies inside one tile
+                const uint32_t tile = sp * 2u + (tid >> 8);
+                if (lane == 0 && wcnt && tile < P.ntiles) atomicAdd(&P.tile_prefix[tile], wcnt);
+                mine += __popc(nib);
             }
-            // eight neighbouring threads make one bitmap word
-            uint32_t word = nib << ((lane & 7u) * 4u);
-            word |= __shfl_xor_sync(FULL, word, 1);
-            word |= __shfl_xor_sync(FULL, word, 2);
-            word |= __shfl_xor_sync(FULL, word, 4);
-            const uint32_t widx = sp * (LT_SPAN / 32u) + (tid >> 3);
-            if ((lane & 7u) == 0u && widx < P.ntiles * 32u) P.bitmap[widx] = word;
-            const uint32_t wcnt = warp_sum(__popc(nib));                     // a warp lies inside one tile
-            const uint32_t tile = sp * 2u + (tid >> 8);
-            if (lane == 0 && wcnt && tile < P.ntiles) atomicAdd(&P.tile_prefix[tile], wcnt);
-            mine += __popc(nib);
         }
     }
     {
@@ -323,7 +400,9 @@ __global__ void __launch_bounds__(LT_THREADS, LT_BLOCKS_PER_SM) layer_topk_kerne
         lt_block_excl_scan(mine, S.wtot, &total);
         if (tid == 0) P.block_tot[blockIdx.x] = total;
     }
+    LT_STAMP(9);
     if (!grid_barrier(gb, &S.flag)) return;
+    LT_STAMP(10);
 
     // ---------------- per-tile counts -> prefix counts (each block its own tiles) -------------------------
     if (tid < 32) {
@@ -365,6 +444,8 @@ __global__ void __launch_bounds__(LT_THREADS, LT_BLOCKS_PER_SM) layer_topk_kerne
             }
         }
     }
+    LT_STAMP(11);
+#undef LT_STAMP
     span_end(P.spans);
 }
 

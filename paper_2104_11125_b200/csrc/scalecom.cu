@@ -124,13 +124,17 @@ cudaError_t launch_chunk(const scalecom_ctx* c, const ChunkParams& P) {
 int ensure_layer_ws(scalecom_ctx* c) {
     if (c->lt_ws) return SCALECOM_OK;
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, layer_topk_kernel<true>, LT_THREADS, sizeof(LayerTopkShared)) !=
+    if (cudaFuncSetAttribute(layer_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(sizeof(LayerTopkShared))) != cudaSuccess ||
+        cudaFuncSetAttribute(layer_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             int(sizeof(LayerTopkShared))) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, layer_topk_kernel<true>, LT_THREADS, sizeof(LayerTopkShared)) !=
             cudaSuccess || occ < 1)
         return SCALECOM_ERR_CUDA;
     if (occ > LT_BLOCKS_PER_SM) occ = LT_BLOCKS_PER_SM;
     c->lt_blocks = uint32_t(c->sms * occ);
     const size_t nl = c->nlayers;
-    c->lt_bytes = nl * LT_BINS * 4 + nl * 16 + 256 + size_t(c->lt_blocks) * 4;
+    c->lt_bytes = nl * LT_ROW * 4 + nl * 16 + 256 + size_t(c->lt_blocks) * 4;
     if (cudaMalloc(&c->lt_ws, c->lt_bytes) != cudaSuccess) {
         cudaGetLastError();
         c->lt_ws = nullptr;
@@ -151,9 +155,9 @@ LayerTopkParams make_layer_params(const scalecom_ctx* c, const float* g, const f
     P.layer_off = c->layer_tab;
     P.layer_k0 = c->layer_tab + (nl + 1);
     P.ghist = reinterpret_cast<uint32_t*>(base);
-    P.lstate = reinterpret_cast<uint4*>(base + nl * LT_BINS * 4);
-    P.tie_flag = reinterpret_cast<uint32_t*>(base + nl * LT_BINS * 4 + nl * 16);
-    P.block_tot = reinterpret_cast<uint32_t*>(base + nl * LT_BINS * 4 + nl * 16 + 256);
+    P.lstate = reinterpret_cast<uint4*>(base + nl * LT_ROW * 4);
+    P.tie_flag = reinterpret_cast<uint32_t*>(base + nl * LT_ROW * 4 + nl * 16);
+    P.block_tot = reinterpret_cast<uint32_t*>(base + nl * LT_ROW * 4 + nl * 16 + 256);
     P.bitmap = c->bitmap; P.tile_prefix = c->tile_prefix; P.ntiles = c->ntiles;
     P.ctrl = c->ctrl;
     P.barrier = c->barrier + 16;               // its own arrival counter (its grid differs from the other selectors')

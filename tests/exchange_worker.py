@@ -1,6 +1,6 @@
 """One rank of a learner-per-process job, run as a child process by test_exchange.py.
 
-usage: exchange_worker.py <cpu|gpu> <topk|chunk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
+usage: exchange_worker.py <cpu|gpu> <topk|chunk|layer_topk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
 
 Every rank generates all learners' seeded inputs, takes the learner of its own rank through
 multi.LearnerRank, and checks each step's index list, reduced values, its learner's memory and
@@ -28,12 +28,15 @@ from paper_2104_11125_b200 import binding, multi, workloads  # noqa: E402
 class OracleEngine:
     """Test-only stand-in with the three calls LearnerRank makes, on CPU tensors."""
 
-    def __init__(self, d, k, beta, lr, selector):
-        self.d, self.k, self.beta, self.lr, self.selector = d, k, beta, lr, selector
+    def __init__(self, d, k, beta, lr, selector, layers):
+        self.d, self.k, self.beta, self.lr, self.selector, self.layers = d, k, beta, lr, selector, layers
 
     def select(self, g, m, out_idx):
         acc = oracle.accumulate(g.numpy(), m.numpy())
-        idx, _ = (oracle.chunk_select if self.selector == "chunk" else oracle.topk)(acc, self.k)
+        if self.selector == "layer_topk":
+            idx, _ = oracle.layer_topk(acc, *self.layers)
+        else:
+            idx, _ = (oracle.chunk_select if self.selector == "chunk" else oracle.topk)(acc, self.k)
         out_idx.copy_(torch.from_numpy(idx))
 
     def compress(self, g, m, idx, out):
@@ -53,13 +56,22 @@ def main():
     rank, world = dist.get_rank(), dist.get_world_size()
     w = workloads.TINY.scaled(d, world)
     k, beta, lr = w.k, w.beta, w.lr
+    layers = None
+    if selector == "layer_topk":                     # five layers of uneven size and rate, the first sent whole
+        sizes = [97, d // 3, 1, d // 5, 0]
+        sizes[4] = d - sum(sizes)
+        keep = [97, max(1, d // 300), 1, max(1, d // 1000), 0]
+        keep[4] = k - sum(keep)
+        assert 1 <= keep[4] <= sizes[4]
+        layers = (sizes, keep)
     dev = torch.device("cuda", 0) if mode == "gpu" else torch.device("cpu")
     if mode == "gpu":
         torch.cuda.set_device(dev)
-        node = multi.LearnerRank(d, k, beta, lr,
-                                 selector=binding.SELECTOR_CHUNK if selector == "chunk" else binding.SELECTOR_TOPK)
+        node = multi.LearnerRank(d, k, beta, lr, layers=layers,
+                                 selector={"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
+                                           "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
     else:
-        node = multi.LearnerRank(d, k, beta, lr, engine=OracleEngine(d, k, beta, lr, selector), device=dev)
+        node = multi.LearnerRank(d, k, beta, lr, engine=OracleEngine(d, k, beta, lr, selector, layers), device=dev)
     prof = workloads.profile(w, dev)
     m_o = [x.cpu().numpy().copy() for x in workloads.initial_memory(w, dev)]
     th_o = workloads.initial_weights(w, dev).cpu().numpy().copy()
@@ -73,7 +85,8 @@ def main():
         if mode == "gpu":
             torch.cuda.synchronize()
             assert node.engine.status() == binding.OK
-        idx_o, val_o, _ = oracle.step(g_all, m_o, th_o, t, k, beta, lr, want_gathered=False, selector=selector)
+        idx_o, val_o, _ = oracle.step(g_all, m_o, th_o, t, k, beta, lr, want_gathered=False,
+                                      selector="topk" if selector == "layer_topk" else selector, layers=layers)
         assert np.array_equal(idx.cpu().numpy(), idx_o), "step %d rank %d: index lists differ" % (t, rank)
         assert np.array_equal(val.cpu().numpy(), val_o), "step %d rank %d: reduced values differ" % (t, rank)
         assert np.array_equal(mem.cpu().numpy(), m_o[rank]), "step %d rank %d: memory differs" % (t, rank)

@@ -32,14 +32,15 @@ def run_ranks(world, mode, selector, d, steps, timeout=240):
         assert "rank %d ok" % rank in out
 
 
-@pytest.mark.parametrize("world,selector", [(2, "topk"), (3, "topk"), (2, "chunk")])
+@pytest.mark.parametrize("world,selector", [(2, "topk"), (3, "topk"), (2, "chunk"), (2, "layer_topk")])
 def test_protocol_over_gloo_matches_single_process_step(world, selector):
     # 2 * world + 1 steps: every rank leads at least twice
     run_ranks(world, "cpu", selector, 40_003, 2 * world + 1)
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("world,selector,d", [(2, "topk", 262_147), (3, "topk", 1_048_583), (3, "chunk", 262_147)])
+@pytest.mark.parametrize("world,selector,d", [(2, "topk", 262_147), (3, "topk", 1_048_583), (3, "chunk", 262_147),
+                                                (2, "layer_topk", 262_147)])
 def test_ranks_sharing_a_device_match_single_process_step(world, selector, d):
     run_ranks(world, "gpu", selector, d, 2 * world + 1, timeout=400)
 

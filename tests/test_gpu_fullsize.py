@@ -222,3 +222,74 @@ def test_layer_rates_full_size_resnet50():
     w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
     paths = workload_case(w2, 2, DEV, selector="chunk", layers=(sizes, keep))
     assert paths == [3, 3]
+
+
+def test_layer_topk_full_size_resnet50():
+    """Exact top-k per tensor with the per-layer rates of Section 4 on the full ResNet-50-shaped vector,
+    every element against the oracle."""
+    from tests.parity import workload_case
+    from paper_2104_11125_b200 import binding
+    w = W.RESNET50
+    sizes, keep = W.resnet50_layer_keep(w)
+    w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
+    paths = workload_case(w2, 2, DEV, selector="layer_topk", layers=(sizes, keep))
+    assert paths == [binding.PATH_LAYER_TOPK] * 2
+
+
+def test_layer_topk_largest_vector_one_layer_and_many():
+    """The per-layer exact selector at d = 2^31 - 1: with one layer the result is Eq. 2 on the whole vector
+    (checked by the threshold property on every coordinate); with 2048 layers, a sample of layers is compared
+    with the oracle run on the layer alone."""
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2 ** 30:
+        pytest.skip("needs ~30 GB of free device memory")
+    d, k = 2 ** 31 - 1, 100_000
+    g = torch.empty(d, device=DEV, dtype=torch.float32)
+    gen = torch.Generator(device=DEV).manual_seed(77)
+    step = 1 << 28
+    for a in range(0, d, step):
+        g[a:min(d, a + step)].normal_(generator=gen)
+    g[d - 1] = 50.0                                           # the last coordinate must be found
+    m = torch.zeros(d, device=DEV)
+    idx = torch.empty(k, device=DEV, dtype=torch.int32)
+    key = g.view(torch.int32) & 0x7FFFFFFF                    # m = 0: acc = g exactly
+    with sc.Context(d, 1, k, 1.0, 0.0) as ctx:
+        ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_LAYER_TOPK)
+        ctx.set_layers([d], [k])
+        ctx.select(g, m, idx)
+        torch.cuda.synchronize()
+        assert ctx.status() == 0 and ctx.query(binding.Q_LAST_TOPK_PATH) == binding.PATH_LAYER_TOPK
+        il = idx.long()
+        assert bool((il[1:] > il[:-1]).all()) and int(il[0]) >= 0 and int(il[-1]) == d - 1
+        sel_keys = key[il]
+        tau = int(sel_keys.min())
+        n_above = int((key > tau).sum())
+        n_at = int((key == tau).sum())
+        assert n_above < k <= n_above + n_at                  # tau is the k-th largest key
+        assert int((sel_keys > tau).sum()) == n_above         # everything above the threshold is in
+        ties = torch.nonzero(key == tau).flatten()            # among equals, the lowest indices win
+        assert torch.equal(torch.sort(il[sel_keys == tau]).values, ties[:k - n_above])
+        del sel_keys, ties
+        # 2048 layers of (almost) equal size, 48 or 49 kept in each
+        nl = 2048
+        sizes = [d // nl] * (nl - 1) + [d - (d // nl) * (nl - 1)]
+        keep = [k // nl] * nl
+        for i in range(k - sum(keep)):
+            keep[i] += 1
+        ctx.set_layers(sizes, keep)
+        ctx.select(g, m, idx)
+        torch.cuda.synchronize()
+        assert ctx.status() == 0
+        got = idx.cpu().numpy().astype(np.int64)
+        assert np.all(np.diff(got) > 0)
+        offs = np.concatenate([[0], np.cumsum(sizes)])
+        koff = np.concatenate([[0], np.cumsum(keep)])
+        for s in (0, 1, 1023, 2046, 2047):
+            x = g[int(offs[s]):int(offs[s + 1])].cpu().numpy()
+            want, _ = oracle.topk(x, keep[s])
+            assert np.array_equal(got[koff[s]:koff[s + 1]], want.astype(np.int64) + offs[s]), s
+        # every layer holds exactly its share
+        counts = np.diff(np.searchsorted(got, offs))
+        assert np.array_equal(counts, np.asarray(keep))
