@@ -9,34 +9,49 @@
 namespace sc {
 
 // bitmap must be zero on entry.  Entries must be strictly ascending and < d; a violation sets the
-// status word (DEV_INTERNAL) instead of writing out of bounds.
+// status word (DEV_INTERNAL) instead of writing out of bounds (tile_prefix may then hold stale entries:
+// the consumer checks every rank against k).
+// tile_prefix[t] = number of entries below t * TILE.  Entry j is the first one at or past the start of
+// every tile t with idx[j-1] / TILE < t <= idx[j] / TILE, so the thread that holds entry j writes j there:
+// usually zero or one tile; a long run of empty tiles is filled by the whole warp.
 __global__ void __launch_bounds__(256) indices_to_bitmap_kernel(const int32_t* __restrict__ idx, uint32_t k, uint32_t d,
                                                                 uint32_t ntiles, uint32_t* bitmap, uint32_t* tile_prefix,
                                                                 uint32_t* status) {
-    const uint32_t gtid = blockIdx.x * blockDim.x + threadIdx.x, gsize = gridDim.x * blockDim.x;
-    for (uint32_t j = gtid; j < k; j += gsize) {
-        const uint32_t p = uint32_t(idx[j]);
-        const bool ok = p < d && (j == 0 || uint32_t(idx[j - 1]) < p);
-        if (ok) atomicOr(&bitmap[p >> 5], 1u << (p & 31u));
-        else atomicCAS(status, DEV_OK, DEV_INTERNAL);
-    }
-    // selected coordinates before a tile = entries below its first coordinate: a lower bound in the list,
-    // one warp per tile probing 32 positions per round (4-5 dependent rounds instead of log2 k)
-    const uint32_t lane = threadIdx.x & 31u, nwarps = gsize >> 5;
-    for (uint32_t tile = gtid >> 5; tile <= ntiles; tile += nwarps) {
-        const uint64_t p0 = uint64_t(tile) * TILE;
-        uint32_t lo = 0, hi = k;
-        while (lo < hi) {                                    // the answer stays in [lo, hi]; the interval shrinks each round
-            const uint32_t step = (hi - lo + 31u) >> 5;
-            const uint64_t pos = uint64_t(lo) + uint64_t(lane) * step;
-            const bool below = pos < hi && uint64_t(uint32_t(idx[pos])) < p0;
-            const uint32_t c = __popc(__ballot_sync(FULL, below));
-            if (c == 0) { hi = lo; break; }
-            const uint64_t top = uint64_t(lo) + uint64_t(c) * step;
-            lo = lo + (c - 1) * step + 1;
-            hi = top < hi ? uint32_t(top) : hi;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t gsize = gridDim.x * blockDim.x;
+    constexpr uint32_t OWN = 4;                                          // tiles a lane fills by itself
+    for (uint32_t j0 = blockIdx.x * blockDim.x + (threadIdx.x & ~31u); j0 < k; j0 += gsize) {   // warp-uniform
+        const uint32_t j = j0 + lane;
+        uint32_t t_lo = 1, t_hi = 0;                                     // tiles [t_lo, t_hi] get prefix j (empty by default)
+        uint32_t tail_lo = 1, tail_hi = 0;                               // the last entry also fills the tiles after it with k
+        if (j < k) {
+            const uint32_t p = uint32_t(idx[j]);
+            const uint32_t prev = j ? uint32_t(idx[j - 1]) : 0u;
+            const bool ok = p < d && (j == 0 || prev < p);
+            if (ok) {
+                atomicOr(&bitmap[p >> 5], 1u << (p & 31u));
+                t_lo = j ? prev / TILE + 1u : 0u;
+                t_hi = p / TILE;
+                if (j == k - 1) { tail_lo = t_hi + 1u; tail_hi = ntiles; }
+            } else {
+                atomicCAS(status, DEV_OK, DEV_INTERNAL);
+            }
         }
-        if (lane == 0) tile_prefix[tile] = lo;
+#pragma unroll
+        for (int round = 0; round < 2; ++round) {
+            const uint32_t lo = round ? tail_lo : t_lo, hi = round ? tail_hi : t_hi;
+            const uint32_t val = round ? k : j;
+            const uint32_t len = hi >= lo ? hi - lo + 1u : 0u;
+            for (uint32_t q = 0; q < (len < OWN ? len : OWN); ++q) tile_prefix[lo + q] = val;
+            uint32_t longs = __ballot_sync(FULL, len > OWN);
+            while (longs) {                                               // warp-uniform
+                const int src = __ffs(longs) - 1;
+                longs &= longs - 1u;
+                const uint32_t s_lo = __shfl_sync(FULL, lo + OWN, src), s_len = __shfl_sync(FULL, len - OWN, src);
+                const uint32_t s_val = __shfl_sync(FULL, val, src);
+                for (uint32_t q = lane; q < s_len; q += 32u) tile_prefix[s_lo + q] = s_val;
+            }
+        }
     }
 }
 

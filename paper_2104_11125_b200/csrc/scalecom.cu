@@ -686,8 +686,7 @@ int scalecom_compress(scalecom_ctx* c, const float* g, float* m, const int32_t* 
     if (!c->bitmap_zero &&
         cudaMemsetAsync(c->bitmap, 0, size_t(c->ntiles) * 32 * 4, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     c->bitmap_zero = true;
-    const uint32_t for_idx = uint32_t((c->k + 255) / 256), for_tiles = c->ntiles / 8 + 1, cap = uint32_t(c->sms) * 16u;
-    const uint32_t want = for_idx > for_tiles ? for_idx : for_tiles;
+    const uint32_t want = uint32_t((c->k + 255) / 256), cap = uint32_t(c->sms) * 16u;
     indices_to_bitmap_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(idx, uint32_t(c->k), uint32_t(c->d), c->ntiles,
                                                                             c->bitmap, c->tile_prefix, c->ctrl + CT_STATUS);
     if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;

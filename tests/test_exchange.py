@@ -163,3 +163,32 @@ def test_compress_takes_whatever_list_comes_next():
             gathered_o = oracle.learner(g.cpu().numpy(), m_o, idx_o, sel, beta)
             assert np.array_equal(out.cpu().numpy(), gathered_o), it
             assert np.array_equal(m.cpu().numpy(), m_o), it
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,picks", [(3_000_000, [5, 1_500_000, 2_999_999]), (3_000_000, [2_999_999]), (3_000_000, [0]),
+                                     (1025, [1024]), (70_000, list(range(1000, 1040)) + [69_999])])
+def test_compress_with_long_runs_of_empty_tiles(d, picks):
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2104_11125_b200 import binding
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    k, beta = len(picks), 0.25
+    gen = torch.Generator(device=dev).manual_seed(9)
+    g = torch.randn(d, device=dev, generator=gen)
+    m = torch.randn(d, device=dev, generator=gen)
+    m_o = m.cpu().numpy().copy()
+    idx_o = np.asarray(picks, np.int32)
+    sel = np.zeros(d, np.uint8)
+    sel[idx_o] = 1
+    out = torch.full((k,), float("nan"), device=dev)
+    with sc.Context(d, 1, k, beta, 0.01) as ctx:
+        ctx.compress(g, m, torch.from_numpy(idx_o).to(dev), out)
+        torch.cuda.synchronize()
+        assert ctx.status() == binding.OK
+    want = oracle.learner(g.cpu().numpy(), m_o, idx_o, sel, beta)
+    assert np.array_equal(out.cpu().numpy(), want)
+    assert np.array_equal(m.cpu().numpy(), m_o)
