@@ -203,7 +203,9 @@ int scalecom_reset(scalecom_ctx* ctx);
                                             set by scalecom_set_layers -- layer s keeps its keep[s] largest
                                             magnitudes, ties to the lower index (steps and scalecom_select
                                             return BAD_STATE while no layers are set).  Its first launch
-                                            after scalecom_set_layers allocates 8 KB per layer             */
+                                            after scalecom_set_layers allocates 8 KB per layer + d bytes;
+                                            SCALECOM_OPT_FORCE_EXACT_PATH = 1 makes it stream g and m in
+                                            every round instead of collecting the undecided coordinates    */
 #define SCALECOM_OPT_KERNEL_SPANS     7  /* 1: every kernel of a step records the time from its first block's
                                             start to its last block's end on the GPU's nanosecond timer
                                             (two atomics per block); read with scalecom_kernel_span_ms     */
@@ -216,7 +218,8 @@ int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 #define SCALECOM_Q_WORKSPACE_BYTES  1  /* device bytes owned by the handle                                    */
 #define SCALECOM_Q_LAST_TOPK_PATH   2  /* last step's selection path: 0 = sampled pre-filter, 1 = full select,
                                           2 = pre-filter started from the previous step's threshold,
-                                          3 = chunk-wise selector, 4 = exact top-k per layer                  */
+                                          3 = chunk-wise selector, 4 = exact top-k per layer (collecting
+                                          route), 5 = the same by its streaming route                         */
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */

@@ -50,7 +50,7 @@ struct scalecom_ctx {
     uint32_t chunk_blocks = 0;
     void* lt_ws = nullptr;             // scratch of the per-layer exact selector (sized by nlayers), or nullptr
     size_t lt_bytes = 0;
-    uint32_t lt_blocks = 0;
+    uint32_t lt_blocks = 0, lt_seg_cap = 0;
     uint32_t nlayers = 0;              // per-layer rates of the chunk-wise selector (0: one rate for the whole vector)
     uint32_t* layer_tab = nullptr;     // device [2][nlayers + 1]: coordinate offsets, chunk offsets
     uint32_t* one_layer_tab = nullptr; // device {0, d, 0, k}: the whole vector as one layer
@@ -134,7 +134,12 @@ int ensure_layer_ws(scalecom_ctx* c) {
     if (occ > LT_BLOCKS_PER_SM) occ = LT_BLOCKS_PER_SM;
     c->lt_blocks = uint32_t(c->sms * occ);
     const size_t nl = c->nlayers;
-    c->lt_bytes = nl * LT_ROW * 4 + nl * 16 + 256 + size_t(c->lt_blocks) * 4;
+    // a warp's segment of undecided coordinates: an eighth of the coordinates it classifies (a few per cent are
+    // expected); when one overflows the kernel falls back to its streaming route
+    const size_t warps = size_t(c->lt_blocks) * LT_WARPS;
+    c->lt_seg_cap = uint32_t((((size_t(c->d) / 8 + warps - 1) / warps + 31) / 32) * 32);
+    if (c->lt_seg_cap < 128u) c->lt_seg_cap = 128u;
+    c->lt_bytes = align_up(nl * LT_ROW * 4 + nl * 16 + 256 + size_t(c->lt_blocks) * 4, 256) + warps * c->lt_seg_cap * 8;
     if (cudaMalloc(&c->lt_ws, c->lt_bytes) != cudaSuccess) {
         cudaGetLastError();
         c->lt_ws = nullptr;
@@ -156,8 +161,11 @@ LayerTopkParams make_layer_params(const scalecom_ctx* c, const float* g, const f
     P.layer_k0 = c->layer_tab + (nl + 1);
     P.ghist = reinterpret_cast<uint32_t*>(base);
     P.lstate = reinterpret_cast<uint4*>(base + nl * LT_ROW * 4);
-    P.tie_flag = reinterpret_cast<uint32_t*>(base + nl * LT_ROW * 4 + nl * 16);
+    P.ctl = reinterpret_cast<uint32_t*>(base + nl * LT_ROW * 4 + nl * 16);
     P.block_tot = reinterpret_cast<uint32_t*>(base + nl * LT_ROW * 4 + nl * 16 + 256);
+    P.cand = reinterpret_cast<uint2*>(base + align_up(nl * LT_ROW * 4 + nl * 16 + 256 + size_t(c->lt_blocks) * 4, 256));
+    P.seg_cap = c->lt_seg_cap;
+    P.force_stream = c->force_exact;
     P.bitmap = c->bitmap; P.tile_prefix = c->tile_prefix; P.ntiles = c->ntiles;
     P.ctrl = c->ctrl;
     P.barrier = c->barrier + 16;               // its own arrival counter (its grid differs from the other selectors')

@@ -234,6 +234,8 @@ def test_layer_topk_full_size_resnet50():
     w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
     paths = workload_case(w2, 2, DEV, selector="layer_topk", layers=(sizes, keep))
     assert paths == [binding.PATH_LAYER_TOPK] * 2
+    paths = workload_case(w2, 1, DEV, selector="layer_topk", layers=(sizes, keep), force_exact=True)
+    assert paths == [binding.PATH_LAYER_TOPK_STREAM]
 
 
 def test_layer_topk_largest_vector_one_layer_and_many():
@@ -260,7 +262,8 @@ def test_layer_topk_largest_vector_one_layer_and_many():
         ctx.set_layers([d], [k])
         ctx.select(g, m, idx)
         torch.cuda.synchronize()
-        assert ctx.status() == 0 and ctx.query(binding.Q_LAST_TOPK_PATH) == binding.PATH_LAYER_TOPK
+        assert ctx.status() == 0 and ctx.query(binding.Q_LAST_TOPK_PATH) in (binding.PATH_LAYER_TOPK,
+                                                                             binding.PATH_LAYER_TOPK_STREAM)
         il = idx.long()
         assert bool((il[1:] > il[:-1]).all()) and int(il[0]) >= 0 and int(il[-1]) == d - 1
         sel_keys = key[il]

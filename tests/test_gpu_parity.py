@@ -436,15 +436,16 @@ def test_layer_topk_small_cases():
         d, k = sum(sizes), sum(keep)
         g = [_t(rng.standard_normal(d)) for _ in range(3)]
         m0 = [torch.zeros(d, device=DEV) for _ in range(3)]
-        for offset in (0, 1):
+        for offset, force in ((0, False), (1, False), (0, True)):
             paths = p.run_and_compare([g] * 3, m0, torch.linspace(-1, 1, d, device=DEV), k, 0.5, 0.25, offset=offset,
-                                      selector="layer_topk", layers=(sizes, keep), tag="layer top-k %d" % len(sizes))
-            assert all(x == binding_path_layer() for x in paths)
+                                      force_exact=force, selector="layer_topk", layers=(sizes, keep),
+                                      tag="layer top-k %d" % len(sizes))
+            assert all(x in LAYER_PATHS for x in paths)
+            if force:
+                assert all(x == 5 for x in paths)
 
 
-def binding_path_layer():
-    from paper_2104_11125_b200 import binding
-    return binding.PATH_LAYER_TOPK
+LAYER_PATHS = (4, 5)        # binding.PATH_LAYER_TOPK (collecting route), binding.PATH_LAYER_TOPK_STREAM
 
 
 def test_layer_topk_ties_across_the_boundary():
@@ -461,10 +462,48 @@ def test_layer_topk_ties_across_the_boundary():
     g = [_t(base), _t(base * 2), _t(-base)]
     m0 = [torch.zeros(d, device=DEV) for _ in range(3)]
     p = _parity()
-    for offset in (0, 3):
-        paths = p.run_and_compare([g] * 3, m0, None, k, 0.5, 0.25, offset=offset, selector="layer_topk",
-                                  layers=(sizes, keep), tag="layer top-k ties")
-        assert all(x == binding_path_layer() for x in paths)
+    for offset, force in ((0, False), (3, False), (0, True)):
+        paths = p.run_and_compare([g] * 3, m0, None, k, 0.5, 0.25, offset=offset, force_exact=force,
+                                  selector="layer_topk", layers=(sizes, keep), tag="layer top-k ties")
+        assert all(x == (5 if force else 4) for x in paths)     # small vector: every undecided coordinate fits its segment
+
+
+def test_layer_topk_overflowing_segments_fall_back_to_streaming():
+    """A large constant layer: every coordinate of it is undecided after the first digit, the warps' segments
+    overflow, and the kernel has to clear the rows and run its streaming route."""
+    rng = np.random.default_rng(47)
+    sizes = [200_000, 2_000_000, 300_000, 500_001]
+    keep = [2000, 12_345, 300_000, 77]
+    d, k = sum(sizes), sum(keep)
+    base = rng.standard_normal(d).astype(np.float32)
+    base[200_000:2_200_000] = -0.375
+    g = [_t(base), _t(base * 3)]
+    m0 = [torch.zeros(d, device=DEV) for _ in range(2)]
+    paths = _parity().run_and_compare([g] * 2, m0, None, k, 0.5, 0.25, selector="layer_topk", layers=(sizes, keep),
+                                      tag="layer top-k overflow")
+    assert paths == [5, 5]
+
+
+def test_layer_topk_small_ties_in_the_collecting_route():
+    """A few exact duplicates of the would-be threshold inside ordinary layers: the collecting route has to
+    split them by offset (lowest index first) without falling back."""
+    rng = np.random.default_rng(43)
+    sizes = [40_000, 60_000, 30_000]
+    keep = [400, 150, 3000]
+    d, k = sum(sizes), sum(keep)
+    base = rng.standard_normal(d).astype(np.float32)
+    off = 0
+    for sz, kp in zip(sizes, keep):
+        mags = np.sort(np.abs(base[off:off + sz]))[::-1]
+        thr = mags[kp - 1]                                      # the kp-th largest magnitude of the layer
+        spots = off + rng.choice(sz, size=7, replace=False)
+        base[spots] = thr * np.where(rng.random(7) < 0.5, 1.0, -1.0).astype(np.float32)
+        off += sz
+    g = [_t(base), _t(base), _t(base)]
+    m0 = [torch.zeros(d, device=DEV) for _ in range(3)]
+    paths = _parity().run_and_compare([g], m0, None, k, 0.5, 0.25, selector="layer_topk", layers=(sizes, keep),
+                                      tag="layer top-k planted ties")
+    assert paths == [4]
 
 
 def test_layer_topk_needs_layers():
@@ -498,4 +537,6 @@ def test_layer_topk_resnet50_rule():
     sizes, keep = W.resnet50_layer_keep(w)
     w2 = W.Workload(w.name + "+layers", w.wid, w.kind, w.n, w.d, sum(keep), w.beta, w.lr, w.steps, w.c)
     paths = _parity().workload_case(w2, 3, DEV, selector="layer_topk", layers=(sizes, keep))
-    assert all(x == binding_path_layer() for x in paths)
+    assert all(x == 4 for x in paths)                          # ordinary gradients: the collecting route
+    paths = _parity().workload_case(w2, 2, DEV, selector="layer_topk", layers=(sizes, keep), force_exact=True)
+    assert all(x == 5 for x in paths)
