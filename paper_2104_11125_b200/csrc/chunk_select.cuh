@@ -112,10 +112,31 @@ __global__ void __launch_bounds__(CS_THREADS, CS_BLOCKS_PER_SM) chunk_select_ker
         bool have[CS_GROUP];
 #pragma unroll
         for (int g = 0; g < CS_GROUP; ++g) { bk[g] = 0; bi[g] = 0xFFFFFFFFu; have[g] = false; }
-        // rows of 32 coordinates, CS_UNROLL rows of every chunk of the group in flight at a time
         uint32_t longest = 0;
 #pragma unroll
         for (int g = 0; g < CS_GROUP; ++g) longest = max(longest, lo[g + 1] - lo[g]);
+        if (LAYERS && longest <= 32u) {
+            // no chunk longer than a row (the 25X layers: 25 coordinates per chunk; a layer sent whole: one):
+            // one load per chunk and lane, no running best
+            float g1[CS_GROUP], m1[CS_GROUP];
+#pragma unroll
+            for (int g = 0; g < CS_GROUP; ++g) {
+                const uint32_t p = lo[g] + lane;
+                if (p < lo[g + 1]) { g1[g] = P.g[p]; m1[g] = P.m[p]; }
+            }
+#pragma unroll
+            for (int g = 0; g < CS_GROUP; ++g) {
+                if (j + g >= jend) break;                               // warp-uniform
+                const uint32_t p = lo[g] + lane;
+                const bool in = p < lo[g + 1];
+                const uint32_t key = in ? mag_key(__fadd_rn(m1[g], g1[g])) : 0u;
+                const uint32_t mx = __reduce_max_sync(FULL, key);
+                const uint32_t best_idx = __reduce_min_sync(FULL, (in && key == mx) ? p : 0xFFFFFFFFu);
+                if (lane == 0) P.best[j + g] = composite(mx, best_idx);
+            }
+            return;
+        }
+        // rows of 32 coordinates, CS_UNROLL rows of every chunk of the group in flight at a time
         for (uint32_t off = 0; off < longest; off += 32u * CS_UNROLL) {
             float gv[CS_GROUP][CS_UNROLL], mv[CS_GROUP][CS_UNROLL];
 #pragma unroll
