@@ -13,7 +13,7 @@
 // end with the largest offset that is still kept.
 //
 // Two routes share these rounds:
-//   collecting (the usual one)  round 0 streams g and m (blocks own contiguous ranges of 2048-coordinate
+//   collecting (the usual one)  the first count streams g and m (blocks own contiguous ranges of 2048-coordinate
 //           spans and count in shared memory); a second streaming pass classifies every coordinate against
 //           its layer's first digit: above it -> selected (bitmap word written), equal -> undecided, kept as
 //           (key, index) in a segment owned by the warp; all later rounds run over these few per cent only.
@@ -434,7 +434,7 @@ __global__ void __launch_bounds__(LT_THREADS, LT_BLOCKS_PER_SM) layer_topk_kerne
 #define LT_BARRIER() do { if (!grid_barrier(gb, &S.flag)) return; } while (0)
 #define LT_LOAD() do { if (have) lt_load_state(P, S, lf, ll); } while (0)
     LT_STAMP(0);
-    // ---------------- round 0: first digit of every layer ---------------------------------------------------
+    // ---------------- first digit of every layer --------------------------------------------------------------
     lt_stream_pass<0, VEC>(P, S, span_lo, span_hi, lf);
     LT_STAMP(1);
     LT_BARRIER();
@@ -496,7 +496,7 @@ __global__ void __launch_bounds__(LT_THREADS, LT_BLOCKS_PER_SM) layer_topk_kerne
                 }
             }
         } else {
-            // a segment overflowed: the rows hold part of round 1 and are cleared before the streaming route starts
+            // a segment overflowed: the rows hold part of the second count and are cleared before the streaming route starts
             for (uint32_t s = blockIdx.x; s < P.nl; s += nblocks)
                 for (uint32_t i = tid; i < LT_BINS; i += LT_THREADS) P.ghist[size_t(s) * LT_ROW + i] = 0u;
             LT_BARRIER();

@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
         }
         if (ok) { fast = true; used_hint = attempt == 0; break; }
         st.prefix = 0; st.nbits = 0; st.need = k; st.group = d;
-        if (attempt == 0) SC_BARRIER();                                // every block has judged the pass before it is undone
+        if (attempt == 0) SC_BARRIER();                                // every block has checked the pass before it is undone
     }
     if (P.force_exact) {
         clear_outputs();
