@@ -176,8 +176,11 @@ int scalecom_apply_update(scalecom_ctx* ctx, float* weights, const int32_t* idx,
 /*
  * Wait for the handle's stream and report the device-side status of the steps
  * issued so far: SCALECOM_OK, SCALECOM_ERR_TIMEOUT or SCALECOM_ERR_INTERNAL
- * (after either of which outputs are undefined and the handle refuses further
- * steps until scalecom_reset), or SCALECOM_ERR_CUDA.
+ * (after either of which the handle refuses further steps until scalecom_reset;
+ * the kernels queued behind the one that failed see the status word and do
+ * nothing, so the failing step's outputs, memories and weights are left as they
+ * were, except where INTERNAL was raised by an index that scalecom_compress or
+ * scalecom_reduce_rows skipped), or SCALECOM_ERR_CUDA.
  */
 int scalecom_status(scalecom_ctx* ctx);
 

@@ -50,6 +50,7 @@ struct LearnerParams {
     float* gathered;                       // [n * k] or nullptr
     float* weights;                        // [d] or nullptr (then Algorithm 1 line 12 is not applied here)
     unsigned long long* spans;             // nullptr, or where to accumulate the kernel's time span
+    const uint32_t* status;                // the handle's status word: anything but DEV_OK and the kernel does nothing
 };
 
 // One burst of a thread covers LP_T consecutive tiles x LP_L learners (LP_T * LP_L = LP_UNROLL pairs of
@@ -70,6 +71,8 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
     float* const gathered = ONE ? nullptr : P.gathered;
     const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside a tile
     const uint32_t sh = (tid & 7u) * 4u;           // and its first bit inside that word
+    // a selection kernel that gave up leaves no valid bitmap or prefix counts behind
+    if (ld_relaxed_u32(P.status) != DEV_OK) return;
     span_begin(P.spans);
 
     const uint32_t nsuper = (P.ntiles + LP_T - 1) / LP_T;
@@ -173,7 +176,9 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
 
 // Algorithm 1 line 12 as its own kernel: theta[idx[j]] -= lr * val[j].
 __global__ void __launch_bounds__(256) apply_update_kernel(float* __restrict__ weights, const int32_t* __restrict__ idx,
-                                                           const float* __restrict__ val, uint32_t k, float lr) {
+                                                           const float* __restrict__ val, uint32_t k, float lr,
+                                                           const uint32_t* __restrict__ status) {
+    if (ld_relaxed_u32(status) != DEV_OK) return;                      // no valid index list after a device error
     for (uint32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < k; j += gridDim.x * blockDim.x) {
         const int32_t p = idx[j];
         weights[p] = __fsub_rn(weights[p], __fmul_rn(lr, val[j]));

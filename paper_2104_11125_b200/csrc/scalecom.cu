@@ -313,6 +313,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     lp.gathered = c->gathered;
     lp.weights = (weights && c->fuse_update) ? weights : nullptr;
     lp.spans = span_slot ? span_slot + 2 : nullptr;
+    lp.status = c->ctrl + CT_STATUS;
 
     bool vec_all = true;
     for (int i = 0; i < c->n; ++i) vec_all = vec_all && aligned16(grads[i]) && aligned16(mem[i]);
@@ -353,7 +354,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     if (weights && !c->fuse_update) {
         const uint32_t blocks = uint32_t((c->k + 255) / 256);
         apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, out_idx, out_val,
-                                                                                   uint32_t(c->k), c->lr);
+                                                                                   uint32_t(c->k), c->lr, c->ctrl + CT_STATUS);
         if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
         ++c->launches;
     }
@@ -632,7 +633,8 @@ int scalecom_apply_update(scalecom_ctx* c, float* weights, const int32_t* idx, c
     DeviceGuard guard(c->device);
     if (!guard.ok) return SCALECOM_ERR_CUDA;
     const uint32_t blocks = uint32_t((k + 255) / 256);
-    apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, idx, val, uint32_t(k), lr);
+    apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, idx, val, uint32_t(k), lr,
+                                                                               c->ctrl + CT_STATUS);
     if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     return SCALECOM_OK;
@@ -707,6 +709,7 @@ int scalecom_compress(scalecom_ctx* c, const float* g, float* m, const int32_t* 
     lp.bitmap = c->bitmap; lp.bitmap_clear = c->bitmap; lp.tile_prefix = c->tile_prefix;
     lp.out_val = out_gathered; lp.out_idx = c->scratch_idx;
     lp.gathered = nullptr; lp.weights = nullptr; lp.spans = nullptr;
+    lp.status = c->ctrl + CT_STATUS;
     const float* gp[1] = {g};
     float* mp[1] = {m};
     const cudaError_t e = (aligned16(g) && aligned16(m)) ? launch_learner<16, true, LP_ONE_T, 1, true>(c, 1, gp, mp, lp)

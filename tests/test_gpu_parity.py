@@ -155,30 +155,51 @@ def test_host_buffer_entry_point():
     assert np.array_equal(th.cpu().numpy(), th_o)
 
 
-def test_bounded_wait_expiry_is_reported_and_recoverable():
+@pytest.mark.parametrize("selector", ["topk", "chunk", "layer_topk"])
+def test_bounded_wait_expiry_is_reported_and_recoverable(selector):
     """Failure detection without a GPU fault: with the barrier's iteration bound set to 0 every
-    wait gives up at once, the kernel returns, the status word says TIMEOUT, the handle refuses
-    work until it is reset, and after the reset results are right again."""
+    wait gives up at once, the kernel returns, the status word says TIMEOUT, the kernels that follow it in
+    the step do nothing (outputs and memory untouched), the handle refuses work until it is reset, and after
+    the reset the same handle gives right results again."""
+    import oracle
     import paper_2104_11125_b200 as sc
     from paper_2104_11125_b200 import binding
     w = W.TINY.scaled(200_000)                      # 25 blocks in the selection kernel
     prof = W.profile(w, DEV)
     g = W.gradients(w, 0, DEV, prof)
-    idx = torch.empty(w.k, device=DEV, dtype=torch.int32)
-    val = torch.empty(w.k, device=DEV)
+    idx = torch.full((w.k,), -7, device=DEV, dtype=torch.int32)
+    val = torch.full((w.k,), 3.5, device=DEV)
+    sizes, keep = [w.d // 2, w.d - w.d // 2], [w.k // 4, w.k - w.k // 4]
+    layers = (sizes, keep) if selector == "layer_topk" else None
     with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
-        assert ctx.query(binding.Q_TOPK_BLOCKS) > 1
+        ctx.set_option(binding.OPT_SELECTOR, {"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
+                                              "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
+        if layers:
+            ctx.set_layers(*layers)
         ctx.set_option(binding.OPT_SPIN_LIMIT, 0)
-        m = W.initial_memory(w, DEV)
-        ctx.step(g, m, None, 0, idx, val)
+        m = [torch.full((w.d,), 0.25, device=DEV) for _ in range(w.n)]
+        theta = torch.full((w.d,), 1.5, device=DEV)
+        ctx.step(g, m, theta, 0, idx, val)
         assert ctx.status() == binding.ERR_TIMEOUT
+        assert bool((idx == -7).all()) and bool((val == 3.5).all()) and bool((theta == 1.5).all())
+        assert all(bool((x == 0.25).all()) for x in m)
         with pytest.raises(sc.ScaleComError) as ei:
             ctx.step(g, m, None, 0, idx, val)
         assert ei.value.code == binding.ERR_BAD_STATE
         ctx.set_option(binding.OPT_SPIN_LIMIT, 1 << 22)
         ctx.reset()
         assert ctx.status() == 0
-    _parity().workload_case(w, 2, DEV)              # a fresh handle on the same device is unaffected
+        # the same handle after the reset, against the oracle
+        m_g = W.initial_memory(w, DEV)
+        m_o = [x.cpu().numpy().copy() for x in m_g]
+        ctx.step(g, m_g, None, 0, idx, val)
+        assert ctx.status() == 0
+        idx_o, val_o, _ = oracle.step([x.cpu().numpy() for x in g], m_o, None, 0, w.k, w.beta, w.lr, want_gathered=False,
+                                      selector="topk" if selector == "layer_topk" else selector, layers=layers)
+        assert np.array_equal(idx.cpu().numpy(), idx_o) and np.array_equal(val.cpu().numpy(), val_o)
+        assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(m_g, m_o))
+    if selector == "topk":
+        _parity().workload_case(w, 2, DEV)          # a fresh handle on the same device is unaffected
 
 
 def test_argument_checks_on_device_pointers():
