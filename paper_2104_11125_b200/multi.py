@@ -43,6 +43,7 @@ class LearnerRank:
         self.rank = dist.get_rank(group)
         self.world = dist.get_world_size(group)
         self.d, self.k, self.lr = int(d), int(k), float(lr)
+        self._flat_gather = dist.get_backend(group) == "nccl"
         if engine is None:
             engine = binding.Context(d, 1, k, beta, lr, stream=torch.cuda.current_stream())
             engine.set_option(binding.OPT_SELECTOR, selector)
@@ -69,7 +70,10 @@ class LearnerRank:
         src = leader if self.group is None else dist.get_global_rank(self.group, leader)
         dist.broadcast(self.idx, src=src, group=self.group)
         self.engine.compress(grad, mem, self.idx, self.own)
-        dist.all_gather(list(self.rows.view(self.world, self.k).unbind(0)), self.own, group=self.group)
+        if self._flat_gather:
+            dist.all_gather_into_tensor(self.rows, self.own, group=self.group)
+        else:                                   # (gloo has no flat all-gather)
+            dist.all_gather(list(self.rows.view(self.world, self.k).unbind(0)), self.own, group=self.group)
         self.engine.reduce_rows(self.rows, self.val, self.idx, weights)
         return self.idx, self.val
 
