@@ -54,6 +54,9 @@ def parse_args():
                     help="one-gpu (default, the headline): all n learners of the workload in each GPU's memory; "
                          "learner-per-gpu: every rank is one learner (n = number of ranks), indices broadcast and "
                          "kept values all-gathered over NCCL between the library's calls")
+    ap.add_argument("--exchange", default="collective", choices=["collective", "peer"],
+                    help="learner-per-gpu only: all-gather of the kept values by NCCL (collective) or fused into the "
+                         "compressing kernel as stores into the peers' mapped buffers (peer)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -234,7 +237,7 @@ def run_learner_per_gpu(args):
     mem = torch.zeros(w.d, device=dev, dtype=torch.float32)          # Algorithm 1: memory starts at zero
     flush = torch.empty(64 << 20, device=dev, dtype=torch.float32)  # 256 MB: written between timed intervals
     theta = W.initial_weights(w, dev)
-    node = multi.LearnerRank(w.d, w.k, w.beta, w.lr,
+    node = multi.LearnerRank(w.d, w.k, w.beta, w.lr, exchange=args.exchange,
                              selector=binding.SELECTOR_CHUNK if args.selector == "chunk" else binding.SELECTOR_TOPK)
     ctx = node.engine
 
@@ -290,7 +293,10 @@ def run_learner_per_gpu(args):
             "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "n": world, "d": w.d, "k": w.k, "beta": w.beta, "lr": w.lr,
-                       "parallelism": "learner per GPU: index broadcast + all-gather of kept values (NCCL)",
+                       "parallelism": "learner per GPU: index broadcast (NCCL) + " +
+                                      ("kept values stored into the peers' mapped rows by the compressing kernel, "
+                                       "one-word all-reduce as fence" if args.exchange == "peer"
+                                       else "all-gather of kept values (NCCL)"),
                        "selector": args.selector, "gradient_batches_resident": nb,
                        "l2": "flushed (256 MB written) before every timed step and call",
                        "exchange_bytes_per_rank_per_step": node.exchange_bytes()},

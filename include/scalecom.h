@@ -162,6 +162,21 @@ int scalecom_set_layers(scalecom_ctx* ctx, int32_t nlayers, const int64_t* sizes
  */
 int scalecom_select(scalecom_ctx* ctx, const float* g, const float* m, int32_t* out_idx);
 int scalecom_compress(scalecom_ctx* ctx, const float* g, float* m, const int32_t* idx, float* out_gathered);
+
+/*
+ * scalecom_compress that also sends: besides out_gathered, every kept value is stored, as the pass produces
+ * it, into n_dst further rows dst[0 .. n_dst) -- this rank's row of every rank's gathered-rows buffer, i.e.
+ * the all-gather of the step fused into the kernel as plain stores (the paper's exchange of the k kept values,
+ * Section 4 / Appendix E).
+ *   dst    HOST array of n_dst DEVICE pointers, each to fp32[k]; they may point into other GPUs' memory that
+ *          this device can address (peer access enabled, or a CUDA IPC mapping).  0 <= n_dst <= 64.
+ * The kernel waits for nobody.  Before a destination is read (scalecom_reduce_rows there) its owner must know
+ * that all senders' kernels have finished -- a barrier or any collective after this call on every rank -- and
+ * a row must not be overwritten by the next step while its owner still reads it (two buffers, used in turn).
+ * Errors: those of scalecom_compress; INVALID_ARG for n_dst outside 0..64; NULL_PTR, ALIAS for a bad dst[i].
+ */
+int scalecom_compress_scatter(scalecom_ctx* ctx, const float* g, float* m, const int32_t* idx, float* out_gathered,
+                              float* const* dst, int32_t n_dst);
 int scalecom_reduce_rows(scalecom_ctx* ctx, const float* rows, int32_t n_rows, float* out_val, const int32_t* idx,
                          float* weights);
 

@@ -31,7 +31,7 @@ EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
     "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
-    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance", "scalecom_set_layers", "scalecom_select", "scalecom_compress", "scalecom_reduce_rows",
+    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance", "scalecom_set_layers", "scalecom_select", "scalecom_compress", "scalecom_reduce_rows", "scalecom_compress_scatter",
 )
 STATIC_MAX_D = 1 << 20
 
@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
         L.scalecom_select.argtypes = [vp, vp, vp, vp]
         L.scalecom_compress.restype = ctypes.c_int
         L.scalecom_compress.argtypes = [vp, vp, vp, vp, vp]
+        L.scalecom_compress_scatter.restype = ctypes.c_int
+        L.scalecom_compress_scatter.argtypes = [vp, vp, vp, vp, vp, vp, i32]
         L.scalecom_reduce_rows.restype = ctypes.c_int
         L.scalecom_reduce_rows.argtypes = [vp, vp, i32, vp, vp, vp]
         L.scalecom_strerror.restype = ctypes.c_char_p
@@ -239,6 +241,14 @@ class Context:
     def compress(self, g: torch.Tensor, m: torch.Tensor, idx: torch.Tensor, out_gathered: torch.Tensor) -> None:
         _check(lib().scalecom_compress(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"), self._idx(idx),
                                        _dev_f32(out_gathered, self.k, "out_gathered")), "scalecom_compress")
+
+    def compress_scatter(self, g: torch.Tensor, m: torch.Tensor, idx: torch.Tensor, out_gathered: torch.Tensor,
+                         dst: Sequence[torch.Tensor]) -> None:
+        """compress, with the kept values also stored into every tensor of dst (fp32[k] each, peers' memory allowed)."""
+        ptrs = _ptr_array([_dev_f32(t, self.k, "dst[%d]" % i) for i, t in enumerate(dst)])
+        _check(lib().scalecom_compress_scatter(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"), self._idx(idx),
+                                               _dev_f32(out_gathered, self.k, "out_gathered"),
+                                               ctypes.cast(ptrs, ctypes.c_void_p), len(dst)), "scalecom_compress_scatter")
 
     def reduce_rows(self, rows: torch.Tensor, out_val: torch.Tensor, idx: Optional[torch.Tensor] = None,
                     weights: Optional[torch.Tensor] = None) -> None:

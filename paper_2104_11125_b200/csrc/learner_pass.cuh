@@ -38,6 +38,14 @@ struct PtrTable {
     float* m[N];
 };
 
+// Where else the single-learner form stores its kept values: one row per peer (this rank's row of every
+// rank's gathered-rows buffer, peers' memory included), written with plain stores as the values are produced.
+constexpr int LP_MAX_PEERS = 64;
+struct PeerTable {
+    float* dst[LP_MAX_PEERS];
+    int32_t n;
+};
+
 struct LearnerParams {
     uint32_t d, k, ntiles;
     int32_t n;
@@ -61,7 +69,7 @@ struct LearnerParams {
 // is written, because the bitmap and prefix counts then come from an index list received from elsewhere.
 template <int N, bool VEC, int LP_T, int LP_L, bool ONE = false>
 __global__ void __launch_bounds__(LP_THREADS, ONE ? LP_ONE_BLOCKS_PER_SM : LP_BLOCKS_PER_SM)
-learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P) {
+learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P, const __grid_constant__ PeerTable peers) {
     static_assert(LP_T * LP_L <= LP_UNROLL, "burst shape");
     constexpr bool GUARD = ONE;
     const uint32_t tid = threadIdx.x, lane = lane_id();
@@ -166,7 +174,10 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                     if (((nib[t] >> c) & 1u) && (!GUARD || r < P.k)) {
                         const float v = __fdiv_rn(sum[t][c], P.nf);                           // line 10: one division by n
                         P.out_idx[r] = int32_t(pc[t] + c);
-                        P.out_val[r++] = v;
+                        P.out_val[r] = v;
+                        if (ONE)
+                            for (int q = 0; q < peers.n; ++q) peers.dst[q][r] = v;    // Eq. 3's values, sent as they are made
+                        ++r;
                         if (weights) weights[pc[t] + c] = __fsub_rn(wv[t][c], __fmul_rn(P.lr, v));   // line 12
                     }
             }

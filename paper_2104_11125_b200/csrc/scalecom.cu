@@ -183,7 +183,11 @@ cudaError_t launch_layer_topk(const scalecom_ctx* c, const LayerTopkParams& P) {
 }
 
 template <int N, bool VEC, int T, int L = LP_UNROLL / T, bool ONE = false>
-cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem, const LearnerParams& P) {
+cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem, const LearnerParams& P,
+                           const PeerTable* peers = nullptr) {
+    PeerTable pt;
+    pt.n = 0;
+    if (peers) pt = *peers;
     PtrTable<N> tab;
     for (int i = 0; i < N; ++i) {
         tab.g[i] = i < n ? grads[i] : nullptr;
@@ -192,7 +196,7 @@ cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* gra
     const uint32_t nsuper = (c->ntiles + T - 1) / T;
     const uint32_t want = ONE ? uint32_t(c->sms) * LP_ONE_BLOCKS_PER_SM : c->lp_blocks;
     const uint32_t blocks = want < nsuper ? want : nsuper;
-    learner_pass_kernel<N, VEC, T, L, ONE><<<blocks, LP_THREADS, 0, c->stream>>>(tab, P);
+    learner_pass_kernel<N, VEC, T, L, ONE><<<blocks, LP_THREADS, 0, c->stream>>>(tab, P, pt);
     return cudaGetLastError();
 }
 
@@ -679,7 +683,22 @@ int scalecom_select(scalecom_ctx* c, const float* g, const float* m, int32_t* ou
 }
 
 int scalecom_compress(scalecom_ctx* c, const float* g, float* m, const int32_t* idx, float* out_gathered) {
-    if (!c || !g || !m || !idx || !out_gathered) return SCALECOM_ERR_NULL_PTR;
+    return scalecom_compress_scatter(c, g, m, idx, out_gathered, nullptr, 0);
+}
+
+int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const int32_t* idx, float* out_gathered,
+                              float* const* dst, int32_t n_dst) {
+    if (!c || !g || !m || !idx || !out_gathered || (n_dst > 0 && !dst)) return SCALECOM_ERR_NULL_PTR;
+    if (n_dst < 0 || n_dst > LP_MAX_PEERS) return SCALECOM_ERR_INVALID_ARG;
+    PeerTable peers;
+    peers.n = n_dst;
+    for (int i = 0; i < n_dst; ++i) {
+        if (!dst[i]) return SCALECOM_ERR_NULL_PTR;
+        if (static_cast<const void*>(dst[i]) == g || static_cast<const void*>(dst[i]) == m ||
+            static_cast<const void*>(dst[i]) == idx)
+            return SCALECOM_ERR_ALIAS;
+        peers.dst[i] = dst[i];
+    }
     if (static_cast<const void*>(g) == static_cast<const void*>(m) || static_cast<const void*>(idx) == out_gathered)
         return SCALECOM_ERR_ALIAS;
     if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
@@ -712,8 +731,8 @@ int scalecom_compress(scalecom_ctx* c, const float* g, float* m, const int32_t* 
     lp.status = c->ctrl + CT_STATUS;
     const float* gp[1] = {g};
     float* mp[1] = {m};
-    const cudaError_t e = (aligned16(g) && aligned16(m)) ? launch_learner<16, true, LP_ONE_T, 1, true>(c, 1, gp, mp, lp)
-                                                         : launch_learner<16, false, LP_ONE_T, 1, true>(c, 1, gp, mp, lp);
+    const cudaError_t e = (aligned16(g) && aligned16(m)) ? launch_learner<16, true, LP_ONE_T, 1, true>(c, 1, gp, mp, lp, &peers)
+                                                         : launch_learner<16, false, LP_ONE_T, 1, true>(c, 1, gp, mp, lp, &peers);
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     c->launches += 2;
     return SCALECOM_OK;

@@ -18,6 +18,13 @@ step over the same learners.  The traffic per rank is k indices in and
 world * k values in, independent of d; no kernel waits on another rank -- every
 exchange is a torch.distributed collective between kernel launches.
 
+With exchange="peer" the all-gather is fused into the compressing kernel instead: every rank maps the
+other ranks' gathered-rows buffers (CUDA IPC; the ranks of a node must number the devices alike) and
+scalecom_compress_scatter stores each kept value straight into this rank's row of every buffer while the pass
+runs.  What remains between the calls is a fence -- a one-word all-reduce -- so that nobody reduces rows
+that are still being written; two buffers are used in turn, so that a fast rank's next step cannot overwrite
+rows a slow rank is still reading.  The kernels still wait for nobody.
+
 This module only orders calls; all arithmetic is in the library's kernels.
 """
 from __future__ import annotations
@@ -36,7 +43,7 @@ class LearnerRank:
 
     def __init__(self, d: int, k: int, beta: float, lr: float, group: Optional[dist.ProcessGroup] = None,
                  selector: int = binding.SELECTOR_TOPK, layers: Optional[Tuple[Sequence[int], Sequence[int]]] = None,
-                 engine=None, device: Optional[torch.device] = None):
+                 engine=None, device: Optional[torch.device] = None, exchange: str = "collective"):
         if not dist.is_initialized():
             raise RuntimeError("torch.distributed must be initialised before a LearnerRank is made")
         self.group = group
@@ -56,6 +63,37 @@ class LearnerRank:
         self.own = torch.empty(self.k, dtype=torch.float32, device=dev)
         self.rows = torch.empty(self.world * self.k, dtype=torch.float32, device=dev)
         self.val = torch.empty(self.k, dtype=torch.float32, device=dev)
+        if exchange not in ("collective", "peer"):
+            raise ValueError("exchange must be 'collective' or 'peer'")
+        self.exchange = exchange
+        if exchange == "peer":
+            if not isinstance(self.engine, binding.Context):
+                raise ValueError("exchange='peer' needs the CUDA engine")
+            self._map_peer_rows(dev)
+
+    def _map_peer_rows(self, dev: torch.device) -> None:
+        """Two gathered-rows buffers [2][world][k] per rank, each mapped into every other rank."""
+        from torch.multiprocessing.reductions import reduce_tensor
+        self.rows2 = torch.zeros(2, self.world, self.k, dtype=torch.float32, device=dev)
+        self._flag = torch.zeros(1, dtype=torch.int32, device=dev)
+        torch.cuda.synchronize(dev)
+        if self.world == 1:
+            self.peer_rows = [self.rows2]
+            return
+        handles = [None] * self.world
+        dist.all_gather_object(handles, reduce_tensor(self.rows2), group=self.group)
+        self.peer_rows = []
+        for r, (rebuild, args) in enumerate(handles):
+            self.peer_rows.append(self.rows2 if r == self.rank else rebuild(*args))
+        dist.barrier(group=self.group)                  # everyone has mapped everyone before the first store
+
+    def _fence(self) -> None:
+        """Returns (in stream order) once every rank's kernels issued so far have finished."""
+        if self._flat_gather:                           # NCCL: ordered on the stream, no host wait
+            dist.all_reduce(self._flag, group=self.group)
+        else:
+            torch.cuda.current_stream().synchronize()
+            dist.barrier(group=self.group)
 
     def leader(self, t: int) -> int:
         return int(t) % self.world
@@ -69,6 +107,13 @@ class LearnerRank:
             self.engine.select(grad, mem, self.idx)
         src = leader if self.group is None else dist.get_global_rank(self.group, leader)
         dist.broadcast(self.idx, src=src, group=self.group)
+        if self.exchange == "peer":
+            b = int(t) & 1
+            self.engine.compress_scatter(grad, mem, self.idx, self.own,
+                                         [rows[b, self.rank] for rows in self.peer_rows])
+            self._fence()
+            self.engine.reduce_rows(self.rows2[b].view(-1), self.val, self.idx, weights)
+            return self.idx, self.val
         self.engine.compress(grad, mem, self.idx, self.own)
         if self._flat_gather:
             dist.all_gather_into_tensor(self.rows, self.own, group=self.group)

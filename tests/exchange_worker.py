@@ -1,6 +1,6 @@
 """One rank of a learner-per-process job, run as a child process by test_exchange.py.
 
-usage: exchange_worker.py <cpu|gpu> <topk|chunk|layer_topk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
+usage: exchange_worker.py <cpu|gpu|gpu-peer> <topk|chunk|layer_topk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
 
 Every rank generates all learners' seeded inputs, takes the learner of its own rank through
 multi.LearnerRank, and checks each step's index list, reduced values, its learner's memory and
@@ -8,6 +8,8 @@ its weight replica, bit for bit, against the oracle's single-process step over a
 
 "gpu": the library's kernels on cuda:0 (the ranks share the device; nothing in a kernel waits for
 another rank, the exchanges are gloo collectives between launches).
+"gpu-peer": as "gpu", with the all-gather fused into the compressing kernel (stores into the other processes'
+gathered-rows buffers, mapped with CUDA IPC).
 "cpu": the same orchestration over an engine made of the oracle's pieces, so that leader rotation,
 broadcast source and row order are checked where there is no GPU.
 """
@@ -64,10 +66,13 @@ def main():
         keep[4] = k - sum(keep)
         assert 1 <= keep[4] <= sizes[4]
         layers = (sizes, keep)
+    peer = mode == "gpu-peer"
+    if peer:
+        mode = "gpu"
     dev = torch.device("cuda", 0) if mode == "gpu" else torch.device("cpu")
     if mode == "gpu":
         torch.cuda.set_device(dev)
-        node = multi.LearnerRank(d, k, beta, lr, layers=layers,
+        node = multi.LearnerRank(d, k, beta, lr, layers=layers, exchange="peer" if peer else "collective",
                                  selector={"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
                                            "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
     else:

@@ -46,6 +46,15 @@ def test_ranks_sharing_a_device_match_single_process_step(world, selector, d):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("world,selector,d", [(2, "topk", 262_147), (3, "chunk", 1_048_583)])
+def test_peer_stores_into_mapped_rows_match_single_process_step(world, selector, d):
+    """The all-gather fused into the compressing kernel: the processes map one another's gathered-rows buffers
+    (CUDA IPC on the shared device) and store their kept values there; 2 * world + 2 steps use both buffers
+    of every rank several times."""
+    run_ranks(world, "gpu-peer", selector, d, 2 * world + 2, timeout=400)
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("selector,d,n", [("topk", 300_007, 4), ("chunk", 300_007, 4), ("topk", 5_000_011, 5)])
 def test_pieces_in_one_process_match_oracle_step(selector, d, n):
     """The calls of the taken-apart step, one handle per learner, without any collective."""
@@ -192,3 +201,48 @@ def test_compress_with_long_runs_of_empty_tiles(d, picks):
     want = oracle.learner(g.cpu().numpy(), m_o, idx_o, sel, beta)
     assert np.array_equal(out.cpu().numpy(), want)
     assert np.array_equal(m.cpu().numpy(), m_o)
+
+
+@pytest.mark.gpu
+def test_compress_scatter_writes_every_destination_and_checks_its_arguments():
+    import ctypes
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2104_11125_b200 import binding
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    d, k, beta = 150_001, 1500, 0.3
+    rng = np.random.default_rng(13)
+    gen = torch.Generator(device=dev).manual_seed(21)
+    g = torch.randn(d, device=dev, generator=gen)
+    m = torch.randn(d, device=dev, generator=gen)
+    m_o = m.cpu().numpy().copy()
+    idx_o = np.sort(rng.choice(d, size=k, replace=False)).astype(np.int32)
+    sel = np.zeros(d, np.uint8)
+    sel[idx_o] = 1
+    idx = torch.from_numpy(idx_o).to(dev)
+    own = torch.empty(k, device=dev)
+    rows = torch.full((5, k), float("nan"), device=dev)
+    with sc.Context(d, 1, k, beta, 0.01) as ctx:
+        ctx.compress_scatter(g, m, idx, own, [rows[0], rows[2], rows[4]])
+        torch.cuda.synchronize()
+        assert ctx.status() == binding.OK
+        want = oracle.learner(g.cpu().numpy(), m_o, idx_o, sel, beta)
+        for r in (0, 2, 4):
+            assert np.array_equal(rows[r].cpu().numpy(), want)
+        assert bool(torch.isnan(rows[1]).all()) and bool(torch.isnan(rows[3]).all())
+        assert np.array_equal(own.cpu().numpy(), want) and np.array_equal(m.cpu().numpy(), m_o)
+        # arguments
+        L, h = binding.lib(), ctx._h
+        ptrs = (ctypes.c_void_p * 65)(*([rows[0].data_ptr()] * 65))
+        args = (h, g.data_ptr(), m.data_ptr(), idx.data_ptr(), own.data_ptr())
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 65) == binding.ERR_INVALID_ARG
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), -1) == binding.ERR_INVALID_ARG
+        assert L.scalecom_compress_scatter(*args, None, 2) == binding.ERR_NULL_PTR
+        ptrs[1] = None
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2) == binding.ERR_NULL_PTR
+        ptrs[1] = m.data_ptr()
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2) == binding.ERR_ALIAS
+        assert np.array_equal(m.cpu().numpy(), m_o)            # the rejected calls touched nothing
