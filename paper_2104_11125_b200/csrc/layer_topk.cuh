@@ -307,7 +307,8 @@ __device__ __forceinline__ uint32_t lt_classify_pass(const LayerTopkParams& P, L
             const uint32_t word = lt_word_of(nib);
             const uint32_t widx = sp * (LT_SPAN / 32u) + (tid >> 3);
             if ((lane & 7u) == 0u && widx < P.ntiles * 32u) P.bitmap[widx] = word;
-            // the undecided ones go to the warp's segment
+            // the undecided ones go to the warp's segment (most quad rows of a strongly compressed layer have none)
+            if (__ballot_sync(FULL, und != 0u) == 0u) continue;             // warp-uniform
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const uint32_t bal = __ballot_sync(FULL, (und >> c) & 1u);
