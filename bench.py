@@ -193,7 +193,7 @@ def run_reference(args):
     }))
 
 
-def time_oracle(w, batches_dev, steps=2, selector="topk", layers=None):
+def time_oracle(w, batches_dev, steps=4, selector="topk", layers=None):
     """cpu_baseline leg: the oracle on full-size steps of the bench workload, on this machine's host cores."""
     import numpy as np
     import oracle
