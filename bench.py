@@ -193,21 +193,28 @@ def run_reference(args):
     }))
 
 
-def time_oracle(w, batches_dev, steps=4, selector="topk", layers=None):
-    """cpu_baseline leg: the oracle on full-size steps of the bench workload, on this machine's host cores."""
+def time_oracle(w, batches_dev, selector="topk", layers=None, budget_s=12.0):
+    """cpu_baseline leg: the oracle, as it stands, on this machine's host cores, for about budget_s seconds: full
+    steps of the bench workload where one fits the budget (up to four of them), else steps over the first
+    coordinates of every learner's vectors (the same recipe at a smaller d; not with per-layer rates)."""
     import numpy as np
     import oracle
-    m = [np.zeros(w.d, np.float32) for _ in range(w.n)]
-    th = np.zeros(w.d, np.float32)
+    est = w.n * w.d / 6.5e7                                            # seconds per full step at the oracle's usual rate
+    d_s = w.d if est <= budget_s or layers is not None else max(1 << 20, int(w.d * budget_s / est))
+    k_s = w.k if d_s == w.d else max(1, w.k * d_s // w.d)
+    steps = max(1, min(4, int(budget_s / max(est * d_s / w.d, 1e-9))))
+    m = [np.zeros(d_s, np.float32) for _ in range(w.n)]
+    th = np.zeros(d_s, np.float32)
     dt = 0.0
     for s in range(steps):
-        g = [x.cpu().numpy() for x in batches_dev[s % len(batches_dev)]]
+        g = [np.ascontiguousarray(x[:d_s].cpu().numpy()) for x in batches_dev[s % len(batches_dev)]]
         t0 = time.perf_counter()
-        oracle.step(g, m, th, s, w.k, w.beta, w.lr, want_gathered=False,
+        oracle.step(g, m, th, s, k_s, w.beta, w.lr, want_gathered=False,
                     selector="topk" if selector == "layer_topk" else selector, layers=layers)
         dt += time.perf_counter() - t0
-    return {"value": w.n * w.d * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-            "sample": "%d full steps of the bench workload (n=%d, d=%d, k=%d), %.1f s" % (steps, w.n, w.d, w.k, dt)}
+    what = "full steps of the bench workload" if d_s == w.d else "steps over the first %d coordinates of every vector" % d_s
+    return {"value": w.n * d_s * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+            "sample": "%d %s (n=%d, d=%d, k=%d), %.1f s" % (steps, what, w.n, w.d, w.k, dt)}
 
 
 def run_learner_per_gpu(args):
