@@ -9,10 +9,10 @@
 //   P0  histogram a strided sample of the keys (top 13 bits)
 //   P1  every block derives from the sample a conservative lower bound on the
 //       k-th key (bin b_lo), aiming at slightly more than k survivors.
-//       P0/P1 are skipped when the previous launch of the same handle left a
-//       hint (the bin just below the one of its k-th key; this leader's own from the
-//       last time it led, else the previous step's): a learner's threshold changes
-//       slowly over a training run.  A hint that turns out useless
+//       P0/P1 are skipped when earlier launches of the same handle left a
+//       hint: the bin of this leader's k-th key the last time it led, moved by what the
+//       previous step's leader saw change over the same interval (else the previous
+//       step's bin), minus a margin.  A hint that turns out useless
 //       costs one wasted pass; the step then runs P0/P1 as if there had been none,
 //       and later hints of the handle keep one more bin of distance
 //   P2  stream g, m once.  A survivor (key bin >= b_lo) is appended as (key, idx)
@@ -70,6 +70,7 @@ constexpr uint32_t BCAP = 1024;                                // boundary list 
 
 // ctrl words
 constexpr int CT_CAND = 0, CT_STATUS = 1, CT_PATH = 2, CT_M = 3, CT_BCOUNT = 4, CT_OVERFLOW = 5, CT_HINT = 6, CT_MARGIN = 7;
+constexpr int CT_DRIFT = 21;                                   // (words 8 .. 20 are the phase stamps)
 constexpr int CT_STAMP = 8, CT_NSTAMPS = 13, CT_WORDS = 32;
 // selection paths reported in ctrl[CT_PATH]
 constexpr uint32_t PATH_FAST = 0, PATH_EXACT = 1, PATH_FAST_HINT = 2;
@@ -253,12 +254,20 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
     st.prefix = 0; st.nbits = 0; st.need = k; st.group = d;
     bool fast = false, used_hint = false;
     uint32_t b_lo = 0, M = 0;
-    // bound to start from (bin + 1, 0 = none): what this leader's own vector gave the last time it led
-    // (learners may differ in scale), else what the previous step found
+    // Bound to start from (bin + 1, 0 = none).  The bin of the k-th key is predicted as what this leader's own
+    // vector gave the last time it led (learners may differ in scale) plus the change the previous step's
+    // leader saw over the same interval (the memories grow together while training warms up: without this
+    // term every leader's own value is stale by n steps and the survivors overflow, again and again); a leader
+    // without a value of its own starts from the previous step's.  The bound lies `margin` bins below.
     uint32_t hint = 0;
+    const uint32_t own_prev = (P.use_hint && P.leader_hint) ? __ldcg(P.leader_hint) : 0u;   // bin + 1, 0 = none
     if (!P.force_exact && P.use_hint) {
-        hint = P.leader_hint ? __ldcg(P.leader_hint) : 0u;
-        if (!hint) hint = __ldcg(&P.ctrl[CT_HINT]);
+        const uint32_t prev = __ldcg(&P.ctrl[CT_HINT]);
+        const int32_t margin = 1 + int32_t(__ldcg(&P.ctrl[CT_MARGIN]));
+        int32_t pred = own_prev ? int32_t(own_prev - 1u) + int32_t(__ldcg(&P.ctrl[CT_DRIFT]))
+                                : int32_t(prev) - 1;
+        pred = min(pred, int32_t(NCOARSE) - 1);
+        if (pred > margin) hint = uint32_t(pred - margin) + 1u;
     }
 
     for (int attempt = hint ? 0 : 1; attempt < 2 && !P.force_exact; ++attempt) {
@@ -711,13 +720,13 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
             P.ctrl[CT_CAND] = 0; P.ctrl[CT_OVERFLOW] = 0;
         }
         if (gtid == 0 && P.use_hint) {
-            // one 13-bit bin (4.4 % in magnitude) below the bin of the k-th key just found; two once a hint failed
+            // the 13-bit bin (4.4 % in magnitude) of the k-th key just found, for this leader and for the next step;
+            // later bounds keep one bin of distance, two once a hint has failed
             if (hint && !used_hint) P.ctrl[CT_MARGIN] = 1u;
-            const uint32_t margin = 1u + ((hint && !used_hint) ? 1u : __ldcg(&P.ctrl[CT_MARGIN]));
             const uint32_t cbk = st.nbits >= 13 ? uint32_t(st.prefix >> (st.nbits - 13)) : 0u;
-            const uint32_t next_hint = cbk > margin ? cbk - margin + 1u : 0u;
-            P.ctrl[CT_HINT] = next_hint;
-            if (P.leader_hint) *P.leader_hint = next_hint;
+            if (cbk && own_prev) P.ctrl[CT_DRIFT] = uint32_t(int32_t(cbk) - int32_t(own_prev - 1u));
+            P.ctrl[CT_HINT] = cbk ? cbk + 1u : 0u;
+            if (P.leader_hint) *P.leader_hint = cbk ? cbk + 1u : 0u;
         }
     }
     SC_STAMP(9);

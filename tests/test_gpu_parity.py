@@ -241,10 +241,10 @@ def test_threshold_hint_is_used_then_survives_scale_jumps():
     scales = [1.0, 1.0, 1e-3, 1e-3, 50.0, 50.0]
     jumpy = [[g * sc for g in step] for step, sc in zip(base, scales)]
     paths = p.run_and_compare(jumpy, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.001, w.lr, tag="jumps")
-    # leaders 0,1,2,3,0,1: a step starts from its leader's own last threshold if it has one, else from the
-    # previous step's; the down-jump fails once (step 2), the up-jump once per leader that still
-    # remembers the old scale (steps 4 and 5)
-    assert paths == [0, 2, 0, 2, 0, 0], paths
+    # leaders 0,1,2,3,0,1: a step starts from its leader's own last threshold, moved by what the previous leader
+    # saw change, if it has one, else from the previous step's; the down-jump fails once (step 2), the up-jump
+    # once (step 4): step 5's leader remembers the old scale but also learns how far step 4's leader had to move
+    assert paths == [0, 2, 0, 2, 0, 2], paths
 
 
 # ---- chunk-wise selector (Section 4 / Appendix E) ----------------------------------------------------
