@@ -561,3 +561,19 @@ def test_layer_topk_resnet50_rule():
     assert all(x == 4 for x in paths)                          # ordinary gradients: the collecting route
     paths = _parity().workload_case(w2, 2, DEV, selector="layer_topk", layers=(sizes, keep), force_exact=True)
     assert all(x == 5 for x in paths)
+
+
+def test_long_run_stays_exact_and_mostly_hinted():
+    """120 steps from a cold start: the memories grow, the thresholds rise with them, six learners of different
+    scale take turns.  Every step matches the oracle, and after the first round of leaders the pre-filter
+    starts from a predicted threshold nearly every time."""
+    from paper_2104_11125_b200 import binding
+    w = W.TINY.scaled(150_001, n=6)
+    prof = W.profile(w, DEV)
+    scale = [1.0, 0.3, 3.0, 1.0, 10.0, 0.1]
+    grads = [[g * s for g, s in zip(W.gradients(w, t % 12, DEV, prof), scale)] for t in range(120)]
+    paths = _parity().run_and_compare(grads, W.initial_memory(w, DEV), W.initial_weights(w, DEV), w.k, 0.1, w.lr,
+                                      tag="long run")
+    assert paths[0] == binding.PATH_SAMPLED
+    hinted = sum(p == binding.PATH_HINTED for p in paths[12:])
+    assert hinted >= 0.9 * len(paths[12:]), paths
