@@ -29,8 +29,36 @@ constexpr int LP_BLOCKS_PER_SM = SC_LP_BLOCKS_PER_SM;
 #ifndef SC_ONE_BLOCKS
 #define SC_ONE_BLOCKS 4
 #endif
+#ifndef SC_FEW_T
+#define SC_FEW_T 2
+#endif
+#ifndef SC_FEW_BLOCKS
+#define SC_FEW_BLOCKS 4
+#endif
+#ifndef SC_FEW2_T
+#define SC_FEW2_T 1
+#endif
+#ifndef SC_FEW2_BLOCKS
+#define SC_FEW2_BLOCKS 5
+#endif
 constexpr int LP_ONE_T = SC_ONE_T;                 // tiles per burst of the single-learner form
 constexpr int LP_ONE_BLOCKS_PER_SM = SC_ONE_BLOCKS;
+constexpr int LP_FEW_T = SC_FEW_T;                 // tiles per burst with one learner
+constexpr int LP_FEW_BLOCKS_PER_SM = SC_FEW_BLOCKS;
+#ifndef SC_MID_T
+#define SC_MID_T 1
+#endif
+#ifndef SC_MID_BLOCKS
+#define SC_MID_BLOCKS 3
+#endif
+#ifndef SC_MID_EARLY
+#define SC_MID_EARLY 1
+#endif
+constexpr int LP_MID_T = SC_MID_T;                 // tiles per burst (of four learners) with 4 to 7 learners
+constexpr int LP_MID_BLOCKS_PER_SM = SC_MID_BLOCKS;
+constexpr bool LP_MID_EARLY = SC_MID_EARLY != 0;
+constexpr int LP_FEW2_T = SC_FEW2_T;               // tiles per burst (of two learners) with 2 or 3 learners
+constexpr int LP_FEW2_BLOCKS_PER_SM = SC_FEW2_BLOCKS;
 
 template <int N>
 struct PtrTable {
@@ -67,14 +95,19 @@ struct LearnerParams {
 // ONE: the single-learner form used when every learner has its own device -- n is 1 at compile time, no
 // weights are touched (the reduced values do not exist yet), and ranks are checked against k before a value
 // is written, because the bitmap and prefix counts then come from an index list received from elsewhere.
-template <int N, bool VEC, int LP_T, int LP_L, bool ONE = false>
-__global__ void __launch_bounds__(LP_THREADS, ONE ? LP_ONE_BLOCKS_PER_SM : LP_BLOCKS_PER_SM)
+// MINB: blocks per SM the kernel is compiled for.  EARLY: the first burst of g and m is requested before
+// anything waits on the bitmap.  Few learners per tile want both (occupancy and the early request supply the
+// loads in flight that a burst of 8 learners supplies by itself); with 4 or more learners the later order and
+// 2 blocks per SM measured faster.
+template <int N, bool VEC, int LP_T, int LP_L, bool ONE = false, int MINB = (ONE ? LP_ONE_BLOCKS_PER_SM : LP_BLOCKS_PER_SM),
+          bool EARLY = ONE, bool N1 = ONE>
+__global__ void __launch_bounds__(LP_THREADS, MINB)
 learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P, const __grid_constant__ PeerTable peers) {
     static_assert(LP_T * LP_L <= LP_UNROLL, "burst shape");
     constexpr bool GUARD = ONE;
     const uint32_t tid = threadIdx.x, lane = lane_id();
     const uint32_t d = P.d;
-    const int n = ONE ? 1 : P.n;
+    const int n = N1 ? 1 : P.n;                    // N1: one learner, known when compiling
     float* const weights = ONE ? nullptr : P.weights;
     float* const gathered = ONE ? nullptr : P.gathered;
     const uint32_t wi = tid >> 3;                  // this thread's bitmap word inside a tile
@@ -85,9 +118,8 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
 
     const uint32_t nsuper = (P.ntiles + LP_T - 1) / LP_T;
     for (uint32_t sup = blockIdx.x; sup < nsuper; sup += gridDim.x) {
-        // Single-learner form: the first (only) burst of g and m is requested before anything waits on the
-        // bitmap, so that one memory latency covers both.  With several learners per tile the later order
-        // measured faster (the loads of a burst then issue back to back with nothing else in flight).
+        // EARLY: the first burst of g and m is requested before anything waits on the bitmap, so that one memory
+        // latency covers both.
         uint32_t pc[LP_T], bw[LP_T], tp[LP_T];
 #pragma unroll
         for (int t = 0; t < LP_T; ++t) {
@@ -108,7 +140,7 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                         load_quad_stream<VEC>(tab.m[i0 + u], pc[t], d, mv[t][u]);
                     }
         };
-        if (ONE) load_burst(0);
+        if (EARLY) load_burst(0);
 
         // per tile: selection bits of this thread's four coordinates and the rank of the first selected one
         uint32_t nib[LP_T], rank0[LP_T];
@@ -141,7 +173,7 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
 
         float sum[LP_T][4];
         for (int i0 = 0; i0 < n; i0 += LP_L) {
-            if (!ONE || i0 > 0) load_burst(i0);
+            if (!EARLY || i0 > 0) load_burst(i0);
 #pragma unroll
             for (int t = 0; t < LP_T; ++t)
 #pragma unroll

@@ -182,7 +182,8 @@ cudaError_t launch_layer_topk(const scalecom_ctx* c, const LayerTopkParams& P) {
                                        dim3(LT_THREADS), args, sizeof(LayerTopkShared), c->stream);
 }
 
-template <int N, bool VEC, int T, int L = LP_UNROLL / T, bool ONE = false>
+template <int N, bool VEC, int T, int L = LP_UNROLL / T, bool ONE = false,
+          int MINB = (ONE ? LP_ONE_BLOCKS_PER_SM : LP_BLOCKS_PER_SM), bool EARLY = ONE, bool N1 = ONE>
 cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem, const LearnerParams& P,
                            const PeerTable* peers = nullptr) {
     PeerTable pt;
@@ -194,23 +195,24 @@ cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* gra
         tab.m[i] = i < n ? mem[i] : nullptr;
     }
     const uint32_t nsuper = (c->ntiles + T - 1) / T;
-    const uint32_t want = ONE ? uint32_t(c->sms) * LP_ONE_BLOCKS_PER_SM : c->lp_blocks;
+    const uint32_t want = uint32_t(c->sms) * MINB;
     const uint32_t blocks = want < nsuper ? want : nsuper;
-    learner_pass_kernel<N, VEC, T, L, ONE><<<blocks, LP_THREADS, 0, c->stream>>>(tab, P, pt);
+    learner_pass_kernel<N, VEC, T, L, ONE, MINB, EARLY, N1><<<blocks, LP_THREADS, 0, c->stream>>>(tab, P, pt);
     return cudaGetLastError();
 }
 
 // burst shape (tiles x learners) by learner count: few learners take more tiles per burst
-inline int burst_tiles(int n) { return n >= 8 ? 1 : n >= 4 ? 2 : n >= 2 ? 4 : 0; }
+inline int burst_tiles(int n) { return n >= 8 ? 1 : n >= 4 ? 2 : n >= 2 ? 4 : 0; }   // (4 and 0 stand for "2 or 3" and "1")
 
 template <int N, bool VEC>
 cudaError_t launch_learner_t(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem,
                              const LearnerParams& P) {
     switch (burst_tiles(n)) {
         case 1: return launch_learner<N, VEC, 1>(c, n, grads, mem, P);
-        case 2: return launch_learner<N, VEC, 2>(c, n, grads, mem, P);
-        case 4: return launch_learner<N, VEC, 4>(c, n, grads, mem, P);
-        default: return launch_learner<N, VEC, 4, 1>(c, n, grads, mem, P);   // one learner: 8 tiles per burst spill
+        case 2: return launch_learner<N, VEC, LP_MID_T, 4, false, LP_MID_BLOCKS_PER_SM, LP_MID_EARLY>(c, n, grads, mem, P);
+        // few learners: more blocks per SM and the first burst requested early
+        case 4: return launch_learner<N, VEC, LP_FEW2_T, 2, false, LP_FEW2_BLOCKS_PER_SM, true>(c, n, grads, mem, P);
+        default: return launch_learner<N, VEC, LP_FEW_T, 1, false, LP_FEW_BLOCKS_PER_SM, true, true>(c, n, grads, mem, P);
     }
 }
 
