@@ -153,7 +153,10 @@ int scalecom_set_layers(scalecom_ctx* ctx, int32_t nlayers, const int64_t* sizes
  *                      SCALECOM_OPT_SELECTOR).
  *   scalecom_compress  g fp32[d] read only; m fp32[d] updated in place (Eq. 4); idx int32[k] strictly
  *                      ascending, < d (otherwise scalecom_status reports INTERNAL and nothing is written
- *                      out of bounds); out_gathered fp32[k] = (m + g)[idx[j]] written.
+ *                      out of bounds); out_gathered fp32[k] = (m + g)[idx[j]] written.  idx == NULL on the
+ *                      leader: the list is the one this handle's scalecom_select produced in the call just
+ *                      before (nothing else on the handle in between, else BAD_STATE); the selection's own
+ *                      bitmap is used and the list is not read again.
  *   scalecom_reduce_rows  rows fp32[n_rows * k] read only; out_val fp32[k] = (sum over rows, in order) / n_rows
  *                      written.  weights fp32[d], if not NULL, gets Algorithm 1 line 12 in the same kernel:
  *                      weights[idx[j]] -= lr * out_val[j], with idx int32[k] the broadcast list (an entry >= d

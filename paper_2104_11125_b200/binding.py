@@ -238,15 +238,18 @@ class Context:
         _check(lib().scalecom_select(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"), self._idx(out_idx)),
                "scalecom_select")
 
-    def compress(self, g: torch.Tensor, m: torch.Tensor, idx: torch.Tensor, out_gathered: torch.Tensor) -> None:
-        _check(lib().scalecom_compress(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"), self._idx(idx),
+    def compress(self, g: torch.Tensor, m: torch.Tensor, idx: Optional[torch.Tensor], out_gathered: torch.Tensor) -> None:
+        """idx None: the list this handle's select() has just produced."""
+        _check(lib().scalecom_compress(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"),
+                                       None if idx is None else self._idx(idx),
                                        _dev_f32(out_gathered, self.k, "out_gathered")), "scalecom_compress")
 
-    def compress_scatter(self, g: torch.Tensor, m: torch.Tensor, idx: torch.Tensor, out_gathered: torch.Tensor,
+    def compress_scatter(self, g: torch.Tensor, m: torch.Tensor, idx: Optional[torch.Tensor], out_gathered: torch.Tensor,
                          dst: Sequence[torch.Tensor]) -> None:
         """compress, with the kept values also stored into every tensor of dst (fp32[k] each, peers' memory allowed)."""
         ptrs = _ptr_array([_dev_f32(t, self.k, "dst[%d]" % i) for i, t in enumerate(dst)])
-        _check(lib().scalecom_compress_scatter(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"), self._idx(idx),
+        _check(lib().scalecom_compress_scatter(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"),
+                                               None if idx is None else self._idx(idx),
                                                _dev_f32(out_gathered, self.k, "out_gathered"),
                                                ctypes.cast(ptrs, ctypes.c_void_p), len(dst)), "scalecom_compress_scatter")
 

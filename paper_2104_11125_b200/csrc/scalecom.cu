@@ -39,6 +39,7 @@ struct scalecom_ctx {
     // launch geometry
     int sms = 0;
     uint32_t topk_blocks = 0, lp_blocks = 0;
+    mutable bool select_fresh = false; // the bitmap and prefix counts are those of this handle's last scalecom_select
     mutable bool bitmap_zero = false;  // the bitmap holds no bits (scalecom_compress leaves it so; selection kernels do not)
     uint32_t samp_stride = 1, samp_target = 1;
 
@@ -106,6 +107,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 template <bool VEC>
 cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
     c->bitmap_zero = false;
+    c->select_fresh = false;
     void* args[] = {const_cast<TopkParams*>(&P)};
     return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&topk_select_kernel<VEC>), dim3(c->topk_blocks),
                                        dim3(TK_THREADS), args, sizeof(TopkShared), c->stream);
@@ -114,6 +116,7 @@ cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
 template <bool VEC>
 cudaError_t launch_chunk(const scalecom_ctx* c, const ChunkParams& P) {
     c->bitmap_zero = false;
+    c->select_fresh = false;
     void* args[] = {const_cast<ChunkParams*>(&P)};
     const void* fn = P.nl > 1 ? reinterpret_cast<const void*>(&chunk_select_kernel<VEC, true>)
                               : reinterpret_cast<const void*>(&chunk_select_kernel<VEC, false>);
@@ -177,6 +180,7 @@ LayerTopkParams make_layer_params(const scalecom_ctx* c, const float* g, const f
 template <bool VEC>
 cudaError_t launch_layer_topk(const scalecom_ctx* c, const LayerTopkParams& P) {
     c->bitmap_zero = false;
+    c->select_fresh = false;
     void* args[] = {const_cast<LayerTopkParams*>(&P)};
     return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&layer_topk_kernel<VEC>), dim3(c->lt_blocks),
                                        dim3(LT_THREADS), args, sizeof(LayerTopkShared), c->stream);
@@ -227,6 +231,7 @@ cudaError_t launch_learner_n(const scalecom_ctx* c, int n, const float* const* g
 
 int init_workspace(scalecom_ctx* c) {
     c->bitmap_zero = false;
+    c->select_fresh = false;
     if (cudaMemsetAsync(c->ws, 0, c->ctrl_region_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     if (c->chunk_best && cudaMemsetAsync(c->chunk_best, 0, size_t(c->k) * 8, c->stream) != cudaSuccess)
         return SCALECOM_ERR_CUDA;
@@ -681,6 +686,7 @@ int scalecom_select(scalecom_ctx* c, const float* g, const float* m, int32_t* ou
     }
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
+    c->select_fresh = true;
     return SCALECOM_OK;
 }
 
@@ -690,20 +696,20 @@ int scalecom_compress(scalecom_ctx* c, const float* g, float* m, const int32_t* 
 
 int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const int32_t* idx, float* out_gathered,
                               float* const* dst, int32_t n_dst) {
-    if (!c || !g || !m || !idx || !out_gathered || (n_dst > 0 && !dst)) return SCALECOM_ERR_NULL_PTR;
+    if (!c || !g || !m || !out_gathered || (n_dst > 0 && !dst)) return SCALECOM_ERR_NULL_PTR;
     if (n_dst < 0 || n_dst > LP_MAX_PEERS) return SCALECOM_ERR_INVALID_ARG;
     PeerTable peers;
     peers.n = n_dst;
     for (int i = 0; i < n_dst; ++i) {
         if (!dst[i]) return SCALECOM_ERR_NULL_PTR;
         if (static_cast<const void*>(dst[i]) == g || static_cast<const void*>(dst[i]) == m ||
-            static_cast<const void*>(dst[i]) == idx)
+            (idx && static_cast<const void*>(dst[i]) == idx))
             return SCALECOM_ERR_ALIAS;
         peers.dst[i] = dst[i];
     }
-    if (static_cast<const void*>(g) == static_cast<const void*>(m) || static_cast<const void*>(idx) == out_gathered)
+    if (static_cast<const void*>(g) == static_cast<const void*>(m) || (idx && static_cast<const void*>(idx) == out_gathered))
         return SCALECOM_ERR_ALIAS;
-    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
+    if (c->poisoned || (!idx && !c->select_fresh)) return SCALECOM_ERR_BAD_STATE;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SCALECOM_ERR_CUDA;
     if (!c->scratch_idx && cudaMalloc(reinterpret_cast<void**>(&c->scratch_idx), size_t(c->k) * 4) != cudaSuccess) {
@@ -714,13 +720,20 @@ int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const i
     // the received index list -> bitmap and tile prefixes in the handle's workspace
     // (the single-learner pass below zeroes every bitmap word it has read, so only a bitmap that a selection
     // kernel wrote since, or a fresh workspace, has to be cleared here)
-    if (!c->bitmap_zero &&
-        cudaMemsetAsync(c->bitmap, 0, size_t(c->ntiles) * 32 * 4, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
-    c->bitmap_zero = true;
-    const uint32_t want = uint32_t((c->k + 255) / 256), cap = uint32_t(c->sms) * 16u;
-    indices_to_bitmap_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(idx, uint32_t(c->k), uint32_t(c->d), c->ntiles,
-                                                                            c->bitmap, c->tile_prefix, c->ctrl + CT_STATUS);
-    if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+    // idx == NULL: the list is the one this handle's own scalecom_select has just produced, and the bitmap and
+    // prefix counts it left in the workspace are used as they are
+    if (idx) {
+        if (!c->bitmap_zero &&
+            cudaMemsetAsync(c->bitmap, 0, size_t(c->ntiles) * 32 * 4, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+        const uint32_t want = uint32_t((c->k + 255) / 256), cap = uint32_t(c->sms) * 16u;
+        indices_to_bitmap_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(idx, uint32_t(c->k), uint32_t(c->d),
+                                                                                c->ntiles, c->bitmap, c->tile_prefix,
+                                                                                c->ctrl + CT_STATUS);
+        if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+        ++c->launches;
+    }
+    c->bitmap_zero = true;                 // (the pass below leaves it so)
+    c->select_fresh = false;
     // this learner's share of steps 1, 3 and 4: a learner pass over one learner; with n = 1 the
     // "average" it writes is the gathered value itself (x / 1 is exact)
     LearnerParams lp;
@@ -736,7 +749,7 @@ int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const i
     const cudaError_t e = (aligned16(g) && aligned16(m)) ? launch_learner<16, true, LP_ONE_T, 1, true>(c, 1, gp, mp, lp, &peers)
                                                          : launch_learner<16, false, LP_ONE_T, 1, true>(c, 1, gp, mp, lp, &peers);
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
-    c->launches += 2;
+    ++c->launches;
     return SCALECOM_OK;
 }
 

@@ -107,14 +107,16 @@ class LearnerRank:
             self.engine.select(grad, mem, self.idx)
         src = leader if self.group is None else dist.get_global_rank(self.group, leader)
         dist.broadcast(self.idx, src=src, group=self.group)
+        # the leader's handle still holds its selection: no need to hand the list back to it
+        own_list = None if self.rank == leader else self.idx
         if self.exchange == "peer":
             b = int(t) & 1
-            self.engine.compress_scatter(grad, mem, self.idx, self.own,
+            self.engine.compress_scatter(grad, mem, own_list, self.own,
                                          [rows[b, self.rank] for rows in self.peer_rows])
             self._fence()
             self.engine.reduce_rows(self.rows2[b].view(-1), self.val, self.idx, weights)
             return self.idx, self.val
-        self.engine.compress(grad, mem, self.idx, self.own)
+        self.engine.compress(grad, mem, own_list, self.own)
         if self._flat_gather:
             dist.all_gather_into_tensor(self.rows, self.own, group=self.group)
         else:                                   # (gloo has no flat all-gather)

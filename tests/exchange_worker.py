@@ -40,8 +40,11 @@ class OracleEngine:
         else:
             idx, _ = (oracle.chunk_select if self.selector == "chunk" else oracle.topk)(acc, self.k)
         out_idx.copy_(torch.from_numpy(idx))
+        self.last = out_idx.clone()
 
     def compress(self, g, m, idx, out):
+        if idx is None:                                  # the leader: the list of the select() just before
+            idx, self.last = self.last, None
         sel = np.zeros(self.d, np.uint8)
         sel[idx.numpy()] = 1
         out.copy_(torch.from_numpy(oracle.learner(g.numpy(), m.numpy(), idx.numpy(), sel, self.beta)))

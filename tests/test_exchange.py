@@ -246,3 +246,48 @@ def test_compress_scatter_writes_every_destination_and_checks_its_arguments():
         ptrs[1] = m.data_ptr()
         assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2) == binding.ERR_ALIAS
         assert np.array_equal(m.cpu().numpy(), m_o)            # the rejected calls touched nothing
+
+
+@pytest.mark.gpu
+def test_compress_without_a_list_needs_a_fresh_select():
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2104_11125_b200 import binding
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    d, k, beta = 200_003, 2000, 0.2
+    gen = torch.Generator(device=dev).manual_seed(3)
+    g = torch.randn(d, device=dev, generator=gen)
+    m = torch.randn(d, device=dev, generator=gen)
+    m_o = m.cpu().numpy().copy()
+    idx = torch.empty(k, device=dev, dtype=torch.int32)
+    out = torch.empty(k, device=dev)
+    with sc.Context(d, 1, k, beta, 0.01) as ctx:
+        with pytest.raises(sc.ScaleComError) as ei:          # nothing selected yet
+            ctx.compress(g, m, None, out)
+        assert ei.value.code == binding.ERR_BAD_STATE
+        for selector in (binding.SELECTOR_TOPK, binding.SELECTOR_CHUNK):
+            ctx.set_option(binding.OPT_SELECTOR, selector)
+            ctx.select(g, m, idx)
+            ctx.compress(g, m, None, out)
+            torch.cuda.synchronize()
+            assert ctx.status() == binding.OK
+            acc = oracle.accumulate(g.cpu().numpy(), m_o)
+            idx_o, sel = (oracle.topk if selector == binding.SELECTOR_TOPK else oracle.chunk_select)(acc, k)
+            want = oracle.learner(g.cpu().numpy(), m_o, idx_o, sel, beta)
+            assert np.array_equal(idx.cpu().numpy(), idx_o)
+            assert np.array_equal(out.cpu().numpy(), want) and np.array_equal(m.cpu().numpy(), m_o)
+            with pytest.raises(sc.ScaleComError) as ei:      # the selection has been used up
+                ctx.compress(g, m, None, out)
+            assert ei.value.code == binding.ERR_BAD_STATE
+        # a list given explicitly after all that still works (the bitmap was left clean)
+        ctx.select(g, m, idx)
+        other = torch.arange(0, 100 * k, 100, device=dev, dtype=torch.int32)
+        sel = np.zeros(d, np.uint8)
+        sel[other.cpu().numpy()] = 1
+        ctx.compress(g, m, other, out)
+        torch.cuda.synchronize()
+        want = oracle.learner(g.cpu().numpy(), m_o, other.cpu().numpy(), sel, beta)
+        assert np.array_equal(out.cpu().numpy(), want) and np.array_equal(m.cpu().numpy(), m_o)
