@@ -314,7 +314,7 @@ def run_learner_per_gpu(args):
                         "note": "median of 30 calls, CUDA events around each call (about 6 us of event overhead each), L2 flushed before each"},
             "gpu_launches": launches, "clocks": clocks,
         }))
-    node.engine.close()
+    node.close()
     dist.destroy_process_group()
 
 

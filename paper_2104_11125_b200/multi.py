@@ -124,6 +124,16 @@ class LearnerRank:
         self.engine.reduce_rows(self.rows, self.val, self.idx, weights)
         return self.idx, self.val
 
+    def close(self) -> None:
+        """Drop the mappings of the peers' buffers (every rank, together), then the handle."""
+        if getattr(self, "peer_rows", None) is not None and self.world > 1:
+            torch.cuda.synchronize()
+            self.peer_rows = None
+            dist.barrier(group=self.group)              # nobody frees a buffer that a peer still has mapped
+        self.peer_rows = None
+        if isinstance(self.engine, binding.Context):
+            self.engine.close()
+
     def exchange_bytes(self) -> int:
         """Payload that crosses the interconnect per rank and step: the k broadcast indices and the
         (world - 1) foreign rows of the all-gather."""

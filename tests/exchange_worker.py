@@ -100,6 +100,7 @@ def main():
         assert np.array_equal(mem.cpu().numpy(), m_o[rank]), "step %d rank %d: memory differs" % (t, rank)
         assert np.array_equal(theta.cpu().numpy(), th_o), "step %d rank %d: weights differ" % (t, rank)
     assert node.exchange_bytes() == (4 * k * world if world > 1 else 0)
+    node.close()
     dist.barrier()
     dist.destroy_process_group()
     print("rank", rank, "ok")
