@@ -45,7 +45,8 @@ typedef enum scalecom_error {
     SCALECOM_ERR_ALLOC        = -3,  /* host or device allocation failed                */
     SCALECOM_ERR_CUDA         = -4,  /* a CUDA runtime call or a launch failed          */
     SCALECOM_ERR_TIMEOUT      = -5,  /* a bounded device-side wait expired              */
-    SCALECOM_ERR_BAD_STATE    = -6,  /* handle poisoned by an earlier device error      */
+    SCALECOM_ERR_BAD_STATE    = -6,  /* the handle cannot take this call as it stands: poisoned by an earlier
+                                        device error, a per-layer selector without layers, no selection to reuse */
     SCALECOM_ERR_INTERNAL     = -7,  /* a device-side consistency check failed          */
     SCALECOM_ERR_ALIAS        = -8   /* buffers that must be distinct overlap           */
 } scalecom_error;

@@ -1053,7 +1053,7 @@ const char* scalecom_strerror(int code) {
         case SCALECOM_ERR_ALLOC: return "allocation failed";
         case SCALECOM_ERR_CUDA: return "CUDA runtime error";
         case SCALECOM_ERR_TIMEOUT: return "device-side wait timed out";
-        case SCALECOM_ERR_BAD_STATE: return "handle in error state (call scalecom_reset)";
+        case SCALECOM_ERR_BAD_STATE: return "the handle cannot take this call in its present state (after a device error: scalecom_reset)";
         case SCALECOM_ERR_INTERNAL: return "device-side consistency check failed";
         case SCALECOM_ERR_ALIAS: return "buffers overlap";
         default: return "unknown error";
