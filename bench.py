@@ -54,9 +54,11 @@ def parse_args():
                     help="one-gpu (default, the headline): all n learners of the workload in each GPU's memory; "
                          "learner-per-gpu: every rank is one learner (n = number of ranks), indices broadcast and "
                          "kept values all-gathered over NCCL between the library's calls")
-    ap.add_argument("--exchange", default="collective", choices=["collective", "peer"],
-                    help="learner-per-gpu only: all-gather of the kept values by NCCL (collective) or fused into the "
-                         "compressing kernel as stores into the peers' mapped buffers (peer)")
+    ap.add_argument("--exchange", default="collective", choices=["collective", "peer", "peer-flags"],
+                    help="learner-per-gpu only: all-gather of the kept values by NCCL (collective); fused into the "
+                         "compressing kernel as stores into the peers' mapped buffers, a one-word all-reduce as fence "
+                         "(peer); or the same with flag words the reducing kernel waits for instead of the fence "
+                         "(peer-flags; one rank per GPU)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -301,9 +303,11 @@ def run_learner_per_gpu(args):
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "n": world, "d": w.d, "k": w.k, "beta": w.beta, "lr": w.lr,
                        "parallelism": "learner per GPU: index broadcast (NCCL) + " +
-                                      ("kept values stored into the peers' mapped rows by the compressing kernel, "
-                                       "one-word all-reduce as fence" if args.exchange == "peer"
-                                       else "all-gather of kept values (NCCL)"),
+                                      {"peer": "kept values stored into the peers' mapped rows by the compressing kernel, "
+                                               "one-word all-reduce as fence",
+                                       "peer-flags": "kept values and flag words stored into the peers' mapped buffers by the "
+                                                     "compressing kernel, the reducing kernel waits for the flags",
+                                       "collective": "all-gather of kept values (NCCL)"}[args.exchange],
                        "selector": args.selector, "gradient_batches_resident": nb,
                        "l2": "flushed (256 MB written) before every timed step and call",
                        "exchange_bytes_per_rank_per_step": node.exchange_bytes()},

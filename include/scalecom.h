@@ -162,6 +162,11 @@ int scalecom_set_layers(scalecom_ctx* ctx, int32_t nlayers, const int64_t* sizes
  *                      written.  weights fp32[d], if not NULL, gets Algorithm 1 line 12 in the same kernel:
  *                      weights[idx[j]] -= lr * out_val[j], with idx int32[k] the broadcast list (an entry >= d
  *                      is skipped and scalecom_status reports INTERNAL); weights NULL: no update, idx unused.
+ *                      wait_flags NULL: the rows are complete when the kernel starts (stream order, or a fence
+ *                      the caller placed).  wait_flags DEVICE uint32[n_rows] with tag != 0 (n_rows <= 64): row
+ *                      i is read only after wait_flags[i] holds tag (see scalecom_compress_scatter); the wait
+ *                      is bounded by SCALECOM_OPT_SPIN_LIMIT polls per word, after which nothing is written
+ *                      and scalecom_status reports TIMEOUT.
  * Errors (all three): NULL_PTR, ALIAS, BAD_STATE, ALLOC (compress, first call), CUDA; INVALID_ARG for n_rows < 1.
  */
 int scalecom_select(scalecom_ctx* ctx, const float* g, const float* m, int32_t* out_idx);
@@ -177,12 +182,19 @@ int scalecom_compress(scalecom_ctx* ctx, const float* g, float* m, const int32_t
  * The kernel waits for nobody.  Before a destination is read (scalecom_reduce_rows there) its owner must know
  * that all senders' kernels have finished -- a barrier or any collective after this call on every rank -- and
  * a row must not be overwritten by the next step while its owner still reads it (two buffers, used in turn).
- * Errors: those of scalecom_compress; INVALID_ARG for n_dst outside 0..64; NULL_PTR, ALIAS for a bad dst[i].
+ *   flag_dst, tag   NULL / 0: no signalling, as described so far.  Otherwise flag_dst is a HOST array of n_dst
+ *          DEVICE pointers to one 32-bit word each (beside the destination's rows, same addressability) and
+ *          tag != 0: after the kernel's last block is through, tag is stored into every flag_dst[i] with
+ *          release semantics at system scope.  scalecom_reduce_rows given those words and the same tag waits
+ *          for them inside its kernel, so no collective is needed between the two calls.  Tags must differ from
+ *          step to step on the same words (the step number plus one will do).
+ * Errors: those of scalecom_compress; INVALID_ARG for n_dst outside 0..64 or flag_dst with tag 0; NULL_PTR,
+ * ALIAS for a bad dst[i] or flag_dst[i].
  */
 int scalecom_compress_scatter(scalecom_ctx* ctx, const float* g, float* m, const int32_t* idx, float* out_gathered,
-                              float* const* dst, int32_t n_dst);
+                              float* const* dst, int32_t n_dst, uint32_t* const* flag_dst, uint32_t tag);
 int scalecom_reduce_rows(scalecom_ctx* ctx, const float* rows, int32_t n_rows, float* out_val, const int32_t* idx,
-                         float* weights);
+                         float* weights, const uint32_t* wait_flags, uint32_t tag);
 
 /*
  * Algorithm 1 line 12 on its own: theta[idx[j]] <- theta[idx[j]] - lr * val[j]

@@ -93,9 +93,9 @@ def lib() -> ctypes.CDLL:
         L.scalecom_compress.restype = ctypes.c_int
         L.scalecom_compress.argtypes = [vp, vp, vp, vp, vp]
         L.scalecom_compress_scatter.restype = ctypes.c_int
-        L.scalecom_compress_scatter.argtypes = [vp, vp, vp, vp, vp, vp, i32]
+        L.scalecom_compress_scatter.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, ctypes.c_uint32]
         L.scalecom_reduce_rows.restype = ctypes.c_int
-        L.scalecom_reduce_rows.argtypes = [vp, vp, i32, vp, vp, vp]
+        L.scalecom_reduce_rows.argtypes = [vp, vp, i32, vp, vp, vp, vp, ctypes.c_uint32]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -151,6 +151,13 @@ def _dev_f32(t: torch.Tensor, numel: int, name: str) -> int:
     if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
             and t.numel() == numel):
         raise TypeError("%s must be a contiguous CUDA float32 tensor of %d elements" % (name, numel))
+    return t.data_ptr()
+
+
+def _dev_i32(t: torch.Tensor, numel: int, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()
+            and t.numel() == numel):
+        raise TypeError("%s must be a contiguous CUDA int32 tensor of %d elements" % (name, numel))
     return t.data_ptr()
 
 
@@ -245,23 +252,32 @@ class Context:
                                        _dev_f32(out_gathered, self.k, "out_gathered")), "scalecom_compress")
 
     def compress_scatter(self, g: torch.Tensor, m: torch.Tensor, idx: Optional[torch.Tensor], out_gathered: torch.Tensor,
-                         dst: Sequence[torch.Tensor]) -> None:
-        """compress, with the kept values also stored into every tensor of dst (fp32[k] each, peers' memory allowed)."""
+                         dst: Sequence[torch.Tensor], flags: Optional[Sequence[torch.Tensor]] = None, tag: int = 0) -> None:
+        """compress, with the kept values also stored into every tensor of dst (fp32[k] each, peers' memory allowed);
+        with flags (one int32 word per destination) and tag != 0 the kernel stores tag there when it is through."""
         ptrs = _ptr_array([_dev_f32(t, self.k, "dst[%d]" % i) for i, t in enumerate(dst)])
+        fptrs = None
+        if flags is not None:
+            if len(flags) != len(dst):
+                raise ValueError("one flag word per destination")
+            fptrs = ctypes.cast(_ptr_array([_dev_i32(f, 1, "flags[%d]" % i) for i, f in enumerate(flags)]), ctypes.c_void_p)
         _check(lib().scalecom_compress_scatter(self._h, _dev_f32(g, self.d, "g"), _dev_f32(m, self.d, "m"),
                                                None if idx is None else self._idx(idx),
                                                _dev_f32(out_gathered, self.k, "out_gathered"),
-                                               ctypes.cast(ptrs, ctypes.c_void_p), len(dst)), "scalecom_compress_scatter")
+                                               ctypes.cast(ptrs, ctypes.c_void_p), len(dst), fptrs, int(tag)),
+               "scalecom_compress_scatter")
 
     def reduce_rows(self, rows: torch.Tensor, out_val: torch.Tensor, idx: Optional[torch.Tensor] = None,
-                    weights: Optional[torch.Tensor] = None) -> None:
-        """out_val = mean of the rows in row order; with idx and weights also weights[idx] -= lr * out_val."""
+                    weights: Optional[torch.Tensor] = None, wait_flags: Optional[torch.Tensor] = None, tag: int = 0) -> None:
+        """out_val = mean of the rows in row order; with idx and weights also weights[idx] -= lr * out_val; with
+        wait_flags (int32[n_rows]) and tag the kernel reads row i only once wait_flags[i] == tag."""
         n_rows = max(1, rows.numel() // self.k)
         _check(lib().scalecom_reduce_rows(self._h, _dev_f32(rows, n_rows * self.k, "rows"), n_rows,
                                           _dev_f32(out_val, self.k, "out_val"),
                                           None if idx is None else self._idx(idx),
-                                          None if weights is None else _dev_f32(weights, self.d, "weights")),
-               "scalecom_reduce_rows")
+                                          None if weights is None else _dev_f32(weights, self.d, "weights"),
+                                          None if wait_flags is None else _dev_i32(wait_flags, n_rows, "wait_flags"),
+                                          int(tag)), "scalecom_reduce_rows")
 
     def overlap(self, grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor], t: int) -> int:
         """Eq. 5's d between the leader's top-k set and the true top-k set (synchronous)."""

@@ -58,13 +58,36 @@ __global__ void __launch_bounds__(256) indices_to_bitmap_kernel(const int32_t* _
 // val[j] = (rows[0][j] + rows[1][j] + ... + rows[n-1][j]) / n, summed in row order; with weights given,
 // Algorithm 1 line 12 follows in the same thread: theta[idx[j]] -= lr * val[j] (an index >= d sets the status
 // word instead).
-__global__ void __launch_bounds__(256) reduce_rows_kernel(const float* __restrict__ rows, int n, uint32_t k, float nf,
+// wait_flags != nullptr: the rows are being stored by other ranks' kernels; row i may be read once wait_flags[i]
+// holds tag (written there by its sender after all its stores).  Every block waits for all n flags, at most
+// spin_limit polls each; when a wait runs out the status word becomes DEV_TIMEOUT and nothing is written.
+__global__ void __launch_bounds__(256) reduce_rows_kernel(const float* rows, int n, uint32_t k, float nf,
                                                           float* __restrict__ val, const int32_t* __restrict__ idx,
                                                           float* __restrict__ weights, uint32_t d, float lr,
-                                                          uint32_t* status) {
+                                                          uint32_t* status, const uint32_t* wait_flags, uint32_t tag,
+                                                          uint32_t spin_limit) {
+    if (wait_flags) {
+        __shared__ int all_there;
+        if (threadIdx.x == 0) all_there = 1;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            bool there = false;
+            for (uint32_t it = 0; it < spin_limit; ++it) {
+                if (ld_acquire_sys_u32(wait_flags + i) == tag) { there = true; break; }
+                if (ld_relaxed_u32(status) != DEV_OK) break;
+                if (it > 64) __nanosleep(it > 4096 ? 256 : 64);
+            }
+            if (!there) {
+                atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+                all_there = 0;
+            }
+        }
+        __syncthreads();
+        if (!all_there) return;
+    }
     for (uint32_t j = blockIdx.x * blockDim.x + threadIdx.x; j < k; j += gridDim.x * blockDim.x) {
-        float s = rows[j];
-        for (int i = 1; i < n; ++i) s = __fadd_rn(s, rows[size_t(i) * k + j]);
+        float s = __ldcg(&rows[j]);                                      // (L2: the rows may have come from other GPUs)
+        for (int i = 1; i < n; ++i) s = __fadd_rn(s, __ldcg(&rows[size_t(i) * k + j]));
         const float v = __fdiv_rn(s, nf);
         val[j] = v;
         if (weights) {

@@ -69,8 +69,14 @@ struct PtrTable {
 // Where else the single-learner form stores its kept values: one row per peer (this rank's row of every
 // rank's gathered-rows buffer, peers' memory included), written with plain stores as the values are produced.
 constexpr int LP_MAX_PEERS = 64;
+// With tag != 0 the kernel also signals: once its last block is through, flag[q] (one word per destination, next
+// to that destination's rows) receives tag with release semantics at system scope, so that a consumer that has
+// read tag there with acquire semantics may read this rank's row.
 struct PeerTable {
     float* dst[LP_MAX_PEERS];
+    uint32_t* flag[LP_MAX_PEERS];
+    uint32_t* done;                        // this handle's count of finished blocks (zero between launches)
+    uint32_t tag;
     int32_t n;
 };
 
@@ -213,6 +219,19 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
                         if (weights) weights[pc[t] + c] = __fsub_rn(wv[t][c], __fmul_rn(P.lr, v));   // line 12
                     }
             }
+    }
+    if (ONE && peers.tag != 0u) {
+        // every block's stores are ordered before its increment (barrier, then a system-wide fence by the thread
+        // that counts); the block that counts last therefore publishes the flags after all of them
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence_system();
+            if (atomicAdd(peers.done, 1u) == gridDim.x - 1u) {
+                __threadfence_system();
+                for (int q = 0; q < peers.n; ++q) st_release_sys_u32(peers.flag[q], peers.tag);
+                *peers.done = 0u;
+            }
+        }
     }
     span_end(P.spans);
 }

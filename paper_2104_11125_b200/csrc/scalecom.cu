@@ -192,6 +192,8 @@ cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* gra
                            const PeerTable* peers = nullptr) {
     PeerTable pt;
     pt.n = 0;
+    pt.tag = 0u;
+    pt.done = nullptr;
     if (peers) pt = *peers;
     PtrTable<N> tab;
     for (int i = 0; i < N; ++i) {
@@ -691,16 +693,23 @@ int scalecom_select(scalecom_ctx* c, const float* g, const float* m, int32_t* ou
 }
 
 int scalecom_compress(scalecom_ctx* c, const float* g, float* m, const int32_t* idx, float* out_gathered) {
-    return scalecom_compress_scatter(c, g, m, idx, out_gathered, nullptr, 0);
+    return scalecom_compress_scatter(c, g, m, idx, out_gathered, nullptr, 0, nullptr, 0u);
 }
 
 int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const int32_t* idx, float* out_gathered,
-                              float* const* dst, int32_t n_dst) {
+                              float* const* dst, int32_t n_dst, uint32_t* const* flag_dst, uint32_t tag) {
     if (!c || !g || !m || !out_gathered || (n_dst > 0 && !dst)) return SCALECOM_ERR_NULL_PTR;
-    if (n_dst < 0 || n_dst > LP_MAX_PEERS) return SCALECOM_ERR_INVALID_ARG;
+    if (n_dst < 0 || n_dst > LP_MAX_PEERS || (flag_dst && tag == 0u)) return SCALECOM_ERR_INVALID_ARG;
     PeerTable peers;
     peers.n = n_dst;
+    peers.tag = (flag_dst && n_dst > 0) ? tag : 0u;
+    peers.done = c->ctrl + CT_PEER_DONE;
     for (int i = 0; i < n_dst; ++i) {
+        peers.flag[i] = nullptr;
+        if (peers.tag) {
+            if (!flag_dst[i]) return SCALECOM_ERR_NULL_PTR;
+            peers.flag[i] = flag_dst[i];
+        }
         if (!dst[i]) return SCALECOM_ERR_NULL_PTR;
         if (static_cast<const void*>(dst[i]) == g || static_cast<const void*>(dst[i]) == m ||
             (idx && static_cast<const void*>(dst[i]) == idx))
@@ -754,9 +763,9 @@ int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const i
 }
 
 int scalecom_reduce_rows(scalecom_ctx* c, const float* rows, int32_t n_rows, float* out_val, const int32_t* idx,
-                         float* weights) {
+                         float* weights, const uint32_t* wait_flags, uint32_t tag) {
     if (!c || !rows || !out_val || (weights && !idx)) return SCALECOM_ERR_NULL_PTR;
-    if (n_rows < 1) return SCALECOM_ERR_INVALID_ARG;
+    if (n_rows < 1 || (wait_flags && (tag == 0u || n_rows > LP_MAX_PEERS))) return SCALECOM_ERR_INVALID_ARG;
     if (static_cast<const void*>(rows) == out_val || static_cast<const void*>(weights) == out_val ||
         static_cast<const void*>(weights) == rows || static_cast<const void*>(idx) == out_val)
         return SCALECOM_ERR_ALIAS;
@@ -766,7 +775,7 @@ int scalecom_reduce_rows(scalecom_ctx* c, const float* rows, int32_t n_rows, flo
     const uint32_t want = uint32_t((c->k + 255) / 256), cap = uint32_t(c->sms) * 8u;
     reduce_rows_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(rows, n_rows, uint32_t(c->k), float(n_rows), out_val,
                                                                       idx, weights, uint32_t(c->d), c->lr,
-                                                                      c->ctrl + CT_STATUS);
+                                                                      c->ctrl + CT_STATUS, wait_flags, tag, c->spin_limit);
     if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     return SCALECOM_OK;

@@ -71,6 +71,7 @@ constexpr uint32_t BCAP = 1024;                                // boundary list 
 // ctrl words
 constexpr int CT_CAND = 0, CT_STATUS = 1, CT_PATH = 2, CT_M = 3, CT_BCOUNT = 4, CT_OVERFLOW = 5, CT_HINT = 6, CT_MARGIN = 7;
 constexpr int CT_DRIFT = 21;                                   // (words 8 .. 20 are the phase stamps)
+constexpr int CT_PEER_DONE = 22;                               // finished blocks of a signalling single-learner pass
 constexpr int CT_STAMP = 8, CT_NSTAMPS = 13, CT_WORDS = 32;
 // selection paths reported in ctrl[CT_PATH]
 constexpr uint32_t PATH_FAST = 0, PATH_EXACT = 1, PATH_FAST_HINT = 2;

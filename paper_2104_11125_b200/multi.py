@@ -25,6 +25,12 @@ runs.  What remains between the calls is a fence -- a one-word all-reduce -- so 
 that are still being written; two buffers are used in turn, so that a fast rank's next step cannot overwrite
 rows a slow rank is still reading.  The kernels still wait for nobody.
 
+With exchange="peer-flags" the fence goes too: the compressing kernel, once its last block is through, stores
+the step's tag into a flag word beside its row in every rank's buffer, and the reducing kernel polls its own
+rank's flag words (bounded; TIMEOUT in the handle's status when a sender never arrives) before it reads the
+rows.  The index broadcast is then the only collective of the step.  Here a kernel does wait for other ranks'
+kernels, so the ranks must be on different GPUs.
+
 This module only orders calls; all arithmetic is in the library's kernels.
 """
 from __future__ import annotations
@@ -63,28 +69,39 @@ class LearnerRank:
         self.own = torch.empty(self.k, dtype=torch.float32, device=dev)
         self.rows = torch.empty(self.world * self.k, dtype=torch.float32, device=dev)
         self.val = torch.empty(self.k, dtype=torch.float32, device=dev)
-        if exchange not in ("collective", "peer"):
-            raise ValueError("exchange must be 'collective' or 'peer'")
+        if exchange not in ("collective", "peer", "peer-flags"):
+            raise ValueError("exchange must be 'collective', 'peer' or 'peer-flags'")
         self.exchange = exchange
-        if exchange == "peer":
+        if exchange != "collective":
             if not isinstance(self.engine, binding.Context):
                 raise ValueError("exchange='peer' needs the CUDA engine")
             self._map_peer_rows(dev)
 
     def _map_peer_rows(self, dev: torch.device) -> None:
-        """Two gathered-rows buffers [2][world][k] per rank, each mapped into every other rank."""
+        """Two gathered-rows buffers [2][world][k] per rank and their flag words [2][world], each mapped into
+        every other rank (one allocation: the flags are the tail of the rows' tensor)."""
         from torch.multiprocessing.reductions import reduce_tensor
-        self.rows2 = torch.zeros(2, self.world, self.k, dtype=torch.float32, device=dev)
+        nrow = 2 * self.world * self.k
+        self._shared = torch.zeros(nrow + 2 * self.world, dtype=torch.float32, device=dev)
         self._flag = torch.zeros(1, dtype=torch.int32, device=dev)
         torch.cuda.synchronize(dev)
+
+        def split(buf):
+            return buf[:nrow].view(2, self.world, self.k), buf[nrow:].view(torch.int32).view(2, self.world)
+
+        self.rows2, self.flags2 = split(self._shared)
         if self.world == 1:
-            self.peer_rows = [self.rows2]
+            self.peer_rows, self.peer_flags = [self.rows2], [self.flags2]
             return
         handles = [None] * self.world
-        dist.all_gather_object(handles, reduce_tensor(self.rows2), group=self.group)
-        self.peer_rows = []
+        dist.all_gather_object(handles, reduce_tensor(self._shared), group=self.group)
+        self.peer_rows, self.peer_flags, self._mapped = [], [], []
         for r, (rebuild, args) in enumerate(handles):
-            self.peer_rows.append(self.rows2 if r == self.rank else rebuild(*args))
+            buf = self._shared if r == self.rank else rebuild(*args)
+            self._mapped.append(buf)
+            rows, flags = split(buf)
+            self.peer_rows.append(rows)
+            self.peer_flags.append(flags)
         dist.barrier(group=self.group)                  # everyone has mapped everyone before the first store
 
     def _fence(self) -> None:
@@ -109,12 +126,18 @@ class LearnerRank:
         dist.broadcast(self.idx, src=src, group=self.group)
         # the leader's handle still holds its selection: no need to hand the list back to it
         own_list = None if self.rank == leader else self.idx
-        if self.exchange == "peer":
+        if self.exchange != "collective":
             b = int(t) & 1
-            self.engine.compress_scatter(grad, mem, own_list, self.own,
-                                         [rows[b, self.rank] for rows in self.peer_rows])
-            self._fence()
-            self.engine.reduce_rows(self.rows2[b].view(-1), self.val, self.idx, weights)
+            dst = [rows[b, self.rank] for rows in self.peer_rows]
+            if self.exchange == "peer":
+                self.engine.compress_scatter(grad, mem, own_list, self.own, dst)
+                self._fence()
+                self.engine.reduce_rows(self.rows2[b].view(-1), self.val, self.idx, weights)
+            else:
+                tag = int(t) + 1                        # never 0, new at every step
+                self.engine.compress_scatter(grad, mem, own_list, self.own, dst,
+                                             [flags[b, self.rank:self.rank + 1] for flags in self.peer_flags], tag)
+                self.engine.reduce_rows(self.rows2[b].view(-1), self.val, self.idx, weights, self.flags2[b], tag)
             return self.idx, self.val
         self.engine.compress(grad, mem, own_list, self.own)
         if self._flat_gather:
@@ -128,9 +151,9 @@ class LearnerRank:
         """Drop the mappings of the peers' buffers (every rank, together), then the handle."""
         if getattr(self, "peer_rows", None) is not None and self.world > 1:
             torch.cuda.synchronize()
-            self.peer_rows = None
+            self.peer_rows = self.peer_flags = self._mapped = None
             dist.barrier(group=self.group)              # nobody frees a buffer that a peer still has mapped
-        self.peer_rows = None
+        self.peer_rows = self.peer_flags = None
         if isinstance(self.engine, binding.Context):
             self.engine.close()
 

@@ -1,6 +1,6 @@
 """One rank of a learner-per-process job, run as a child process by test_exchange.py.
 
-usage: exchange_worker.py <cpu|gpu|gpu-peer> <topk|chunk|layer_topk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
+usage: exchange_worker.py <cpu|gpu|gpu-peer|gpu-flags> <topk|chunk|layer_topk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
 
 Every rank generates all learners' seeded inputs, takes the learner of its own rank through
 multi.LearnerRank, and checks each step's index list, reduced values, its learner's memory and
@@ -10,6 +10,8 @@ its weight replica, bit for bit, against the oracle's single-process step over a
 another rank, the exchanges are gloo collectives between launches).
 "gpu-peer": as "gpu", with the all-gather fused into the compressing kernel (stores into the other processes'
 gathered-rows buffers, mapped with CUDA IPC).
+"gpu-flags": as "gpu-peer" without the fence: the reducing kernel waits for flag words the compressing kernels
+set.  Only for a single rank here: kernels of different processes that wait for one another must not share a device.
 "cpu": the same orchestration over an engine made of the oracle's pieces, so that leader rotation,
 broadcast source and row order are checked where there is no GPU.
 """
@@ -59,6 +61,7 @@ def main():
     mode, selector, d, steps = sys.argv[1], sys.argv[2], int(sys.argv[3]), int(sys.argv[4])
     dist.init_process_group("gloo")
     rank, world = dist.get_rank(), dist.get_world_size()
+    assert not (mode == "gpu-flags" and world > 1), "ranks that wait for one another need a GPU each"
     w = workloads.TINY.scaled(d, world)
     k, beta, lr = w.k, w.beta, w.lr
     layers = None
@@ -69,13 +72,13 @@ def main():
         keep[4] = k - sum(keep)
         assert 1 <= keep[4] <= sizes[4]
         layers = (sizes, keep)
-    peer = mode == "gpu-peer"
-    if peer:
+    exchange = {"gpu-peer": "peer", "gpu-flags": "peer-flags"}.get(mode, "collective")
+    if exchange != "collective":
         mode = "gpu"
     dev = torch.device("cuda", 0) if mode == "gpu" else torch.device("cpu")
     if mode == "gpu":
         torch.cuda.set_device(dev)
-        node = multi.LearnerRank(d, k, beta, lr, layers=layers, exchange="peer" if peer else "collective",
+        node = multi.LearnerRank(d, k, beta, lr, layers=layers, exchange=exchange,
                                  selector={"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
                                            "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
     else:

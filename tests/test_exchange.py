@@ -238,13 +238,16 @@ def test_compress_scatter_writes_every_destination_and_checks_its_arguments():
         L, h = binding.lib(), ctx._h
         ptrs = (ctypes.c_void_p * 65)(*([rows[0].data_ptr()] * 65))
         args = (h, g.data_ptr(), m.data_ptr(), idx.data_ptr(), own.data_ptr())
-        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 65) == binding.ERR_INVALID_ARG
-        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), -1) == binding.ERR_INVALID_ARG
-        assert L.scalecom_compress_scatter(*args, None, 2) == binding.ERR_NULL_PTR
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 65, None, 0) == binding.ERR_INVALID_ARG
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), -1, None, 0) == binding.ERR_INVALID_ARG
+        assert L.scalecom_compress_scatter(*args, None, 2, None, 0) == binding.ERR_NULL_PTR
         ptrs[1] = None
-        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2) == binding.ERR_NULL_PTR
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2, None, 0) == binding.ERR_NULL_PTR
         ptrs[1] = m.data_ptr()
-        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2) == binding.ERR_ALIAS
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2, None, 0) == binding.ERR_ALIAS
+        ptrs[1] = rows[1].data_ptr()
+        assert L.scalecom_compress_scatter(*args, ctypes.cast(ptrs, ctypes.c_void_p), 2, ctypes.cast(ptrs, ctypes.c_void_p),
+                                           0) == binding.ERR_INVALID_ARG          # flag words without a tag
         assert np.array_equal(m.cpu().numpy(), m_o)            # the rejected calls touched nothing
 
 
@@ -291,3 +294,93 @@ def test_compress_without_a_list_needs_a_fresh_select():
         torch.cuda.synchronize()
         want = oracle.learner(g.cpu().numpy(), m_o, other.cpu().numpy(), sel, beta)
         assert np.array_equal(out.cpu().numpy(), want) and np.array_equal(m.cpu().numpy(), m_o)
+
+
+@pytest.mark.gpu
+def test_flag_signalled_exchange_single_rank_through_the_orchestration():
+    """exchange="peer-flags" with one rank: the compressing kernel sets the flag word, the reducing kernel that
+    follows it on the stream finds it set.  (Several ranks would need a GPU each.)"""
+    run_ranks(1, "gpu-flags", "topk", 262_147, 5, timeout=300)
+
+
+@pytest.mark.gpu
+def test_flag_signalled_exchange_rank_by_rank_in_one_process():
+    """Four learners' handles in one process, one stream: every compress_scatter stores its row and its flag word
+    into all four gathered-rows buffers; every reduce_rows then waits (finding the flags already set) and sums.
+    Nothing ever waits for a kernel that has not been launched before it."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2104_11125_b200 import binding, workloads
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    n = 4
+    w = workloads.TINY.scaled(400_009, n)
+    d, k, beta, lr = w.d, w.k, w.beta, w.lr
+    prof = workloads.profile(w, dev)
+    mem = workloads.initial_memory(w, dev)
+    m_o = [x.cpu().numpy().copy() for x in mem]
+    theta = [workloads.initial_weights(w, dev) for _ in range(n)]
+    th_o = theta[0].cpu().numpy().copy()
+    ctxs = [sc.Context(d, 1, k, beta, lr) for _ in range(n)]
+    rows = [torch.full((2, n, k), float("nan"), device=dev) for _ in range(n)]        # rank r's two buffers
+    flags = [torch.zeros(2, n, dtype=torch.int32, device=dev) for _ in range(n)]
+    idx = torch.empty(k, device=dev, dtype=torch.int32)
+    own = torch.empty(k, device=dev)
+    val = [torch.empty(k, device=dev) for _ in range(n)]
+    try:
+        for t in range(7):
+            b, tag, leader = t & 1, t + 1, t % n
+            g = workloads.gradients(w, t, dev, prof)
+            ctxs[leader].select(g[leader], mem[leader], idx)
+            for i in range(n):
+                ctxs[i].compress_scatter(g[i], mem[i], None if i == leader else idx, own,
+                                         [rows[r][b, i] for r in range(n)], [flags[r][b, i:i + 1] for r in range(n)], tag)
+            for r in range(n):
+                ctxs[r].reduce_rows(rows[r][b].view(-1), val[r], idx, theta[r], flags[r][b], tag)
+            torch.cuda.synchronize()
+            assert all(c.status() == binding.OK for c in ctxs)
+            idx_o, val_o, G_o = oracle.step([x.cpu().numpy() for x in g], m_o, th_o, t, k, beta, lr)
+            assert np.array_equal(idx.cpu().numpy(), idx_o)
+            for r in range(n):
+                assert np.array_equal(rows[r][b].cpu().numpy(), G_o)
+                assert np.array_equal(val[r].cpu().numpy(), val_o)
+                assert np.array_equal(theta[r].cpu().numpy(), th_o)
+                assert np.array_equal(mem[r].cpu().numpy(), m_o[r])
+                assert flags[r][b].cpu().tolist() == [tag] * n
+    finally:
+        for c in ctxs:
+            c.close()
+
+
+@pytest.mark.gpu
+def test_waiting_for_a_row_that_never_comes_times_out_cleanly():
+    """Failure detection without a GPU fault: a flag word that nothing sets makes the bounded wait of the reducing
+    kernel run out; nothing is written, the status says TIMEOUT, the handle works again after a reset."""
+    import torch
+    from paper_2104_11125_b200 import binding
+    import paper_2104_11125_b200 as sc
+
+    dev = torch.device("cuda", 0)
+    d, k = 50_000, 500
+    rows = torch.ones(3, k, device=dev)
+    flags = torch.tensor([9, 9, 0], dtype=torch.int32, device=dev)          # the third sender never arrives
+    val = torch.full((k,), -1.0, device=dev)
+    with sc.Context(d, 1, k, 0.5, 0.1) as ctx:
+        ctx.set_option(binding.OPT_SPIN_LIMIT, 300)
+        ctx.reduce_rows(rows.view(-1), val, None, None, flags, 9)
+        assert ctx.status() == binding.ERR_TIMEOUT
+        assert bool((val == -1.0).all())
+        with pytest.raises(sc.ScaleComError) as ei:
+            ctx.reduce_rows(rows.view(-1), val, None, None, flags, 9)
+        assert ei.value.code == binding.ERR_BAD_STATE
+        ctx.reset()
+        flags[2] = 9
+        ctx.reduce_rows(rows.view(-1), val, None, None, flags, 9)
+        torch.cuda.synchronize()
+        assert ctx.status() == binding.OK and bool((val == 1.0).all())
+        # argument checks
+        with pytest.raises(sc.ScaleComError) as ei:
+            ctx.reduce_rows(rows.view(-1), val, None, None, flags, 0)
+        assert ei.value.code == binding.ERR_INVALID_ARG
