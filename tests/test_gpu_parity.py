@@ -376,8 +376,9 @@ def test_diagnostics_match_oracle(base, d, n):
         assert ctx.overlap(g, W.initial_memory(w1, DEV), 0) == 0
 
 
+@pytest.mark.parametrize("selector", ["topk", "chunk", "layer_topk"])
 @pytest.mark.parametrize("force_exact", [False, True])
-def test_non_finite_inputs_follow_the_key_order(force_exact):
+def test_non_finite_inputs_follow_the_key_order(force_exact, selector):
     """Keys are the bit patterns of |acc|, so +-Inf rank above every finite value and NaN above Inf,
     deterministically; the rest of the step is plain IEEE arithmetic on both sides."""
     import paper_2104_11125_b200 as sc
@@ -393,12 +394,18 @@ def test_non_finite_inputs_follow_the_key_order(force_exact):
     gd, md, thd = [_t(x) for x in g], [_t(x) for x in m], _t(th)
     idx = torch.empty(k, device=DEV, dtype=torch.int32)
     val = torch.empty(k, device=DEV)
+    layers = ([15_000, 5_000, 20_000], [150, 50, 200]) if selector == "layer_topk" else None
     with sc.Context(d, n, k, 0.5, 0.25) as ctx:
         ctx.set_option(binding.OPT_FORCE_EXACT_PATH, int(force_exact))
+        ctx.set_option(binding.OPT_SELECTOR, {"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
+                                              "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
+        if layers:
+            ctx.set_layers(*layers)
         ctx.step(gd, md, thd, 0, idx, val)
         assert ctx.status() == 0
-    idx_o, val_o, _ = oracle.step(g, m, th, 0, k, 0.5, 0.25)
-    assert {5, 17_000, 39_999} <= set(idx_o.tolist())
+    idx_o, val_o, _ = oracle.step(g, m, th, 0, k, 0.5, 0.25, selector="topk" if selector == "layer_topk" else selector,
+                                  layers=layers)
+    assert {5, 17_000, 39_999} <= set(idx_o.tolist())                # each is the largest key of its chunk or layer too
     assert np.array_equal(idx.cpu().numpy(), idx_o)
     assert np.array_equal(val.cpu().numpy(), val_o, equal_nan=True)
     for a, b in zip(md, m):
