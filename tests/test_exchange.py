@@ -7,12 +7,15 @@ import sys
 
 import pytest
 
+import itertools
+
 HERE = os.path.dirname(os.path.abspath(__file__))
+_launch_no = itertools.count()
 WORKER = os.path.join(HERE, "exchange_worker.py")
 
 
 def run_ranks(world, mode, selector, d, steps, timeout=240):
-    port = 23000 + (os.getpid() * 7 + world * 13 + len(selector)) % 4000
+    port = 23000 + (os.getpid() * 7 + next(_launch_no) * 37) % 4000        # a fresh port for every launch
     procs = []
     for rank in range(world):
         env = dict(os.environ, RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
