@@ -447,10 +447,10 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
         }
     }
     {
-        // candidate segment per warp of the selection grid: room for 4k survivors overall plus slack
+        // candidate segment per warp of the selection grid: room for 6k survivors overall plus slack
         // for uneven spread, never more than the warp's share of the vector
         const int64_t warps = int64_t(c->topk_blocks) * TK_WARPS;
-        int64_t cap = (4 * k + warps - 1) / warps + 32;
+        int64_t cap = (6 * k + warps - 1) / warps + 32;
         const int64_t share = (d + warps - 1) / warps + 32;
         if (cap > share) cap = share;
         c->seg_cap = uint32_t(cap);

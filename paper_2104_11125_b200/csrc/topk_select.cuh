@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
 
     SelState st;
     st.prefix = 0; st.nbits = 0; st.need = k; st.group = d;
-    bool fast = false, used_hint = false;
+    bool fast = false, used_hint = false, hint_overflowed = false;
     uint32_t b_lo = 0, M = 0;
     // Bound to start from (bin + 1, 0 = none).  The bin of the k-th key is predicted as what this leader's own
     // vector gave the last time it led (learners may differ in scale) plus the change the previous step's
@@ -416,7 +416,9 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
 
         // ---------------- P3: locate the k-th composite -------------------------------------------
         M = __ldcg(&P.ctrl[CT_CAND]);
-        bool ok = (M >= k) && __ldcg(&P.ctrl[CT_OVERFLOW]) == 0u;
+        const bool overflowed = __ldcg(&P.ctrl[CT_OVERFLOW]) != 0u;
+        bool ok = (M >= k) && !overflowed;
+        if (attempt == 0) hint_overflowed = overflowed;
         if (ok) {
             find_from_top(P.coarse_win, WIN + 1, k, s);
             const uint32_t cb = s.res[0], above = s.res[1], at = s.res[2];
@@ -721,9 +723,12 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
             P.ctrl[CT_CAND] = 0; P.ctrl[CT_OVERFLOW] = 0;
         }
         if (gtid == 0 && P.use_hint) {
-            // the 13-bit bin (4.4 % in magnitude) of the k-th key just found, for this leader and for the next step;
-            // later bounds keep one bin of distance, two once a hint has failed
-            if (hint && !used_hint) P.ctrl[CT_MARGIN] = 1u;
+            // the 13-bit bin (about 3 % in magnitude) of the k-th key just found, for this leader and for the next
+            // step.  Later bounds keep one bin of distance; two after a hint that left too few survivors, one again
+            // after one that left too many or came close to it (error feedback piles coordinates up just below
+            // the threshold: late in a run one bin holds about k of them)
+            if (hint && !used_hint) P.ctrl[CT_MARGIN] = hint_overflowed ? 0u : 1u;
+            else if (used_hint && M > 3u * k) P.ctrl[CT_MARGIN] = 0u;
             const uint32_t cbk = st.nbits >= 13 ? uint32_t(st.prefix >> (st.nbits - 13)) : 0u;
             if (cbk && own_prev) P.ctrl[CT_DRIFT] = uint32_t(int32_t(cbk) - int32_t(own_prev - 1u));
             P.ctrl[CT_HINT] = cbk ? cbk + 1u : 0u;
