@@ -308,6 +308,10 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
 
     unsigned long long* const span_slot =
         (c->span_timing && c->spans) ? c->spans + 4 * (c->span_steps % scalecom_ctx::EV_RING) : nullptr;
+    // a slot of the ring that already holds an earlier step's span starts from zero again
+    if (span_slot && c->span_steps >= scalecom_ctx::EV_RING &&
+        cudaMemsetAsync(span_slot, 0, 4 * sizeof(unsigned long long), c->stream) != cudaSuccess)
+        return SCALECOM_ERR_CUDA;
     const TopkParams tp = make_topk_params(c, grads[leader], mem[leader], c->leader_hint + leader, true, span_slot);
 
     LearnerParams lp;
