@@ -214,7 +214,12 @@ template <int N, bool VEC>
 cudaError_t launch_learner_t(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem,
                              const LearnerParams& P) {
     switch (burst_tiles(n)) {
-        case 1: return launch_learner<N, VEC, 1>(c, n, grads, mem, P);
+        case 1:
+            // 9 to 14 learners: two bursts of equal size instead of eight and the rest
+            if (N == 16 && n > 8 && n <= 10) return launch_learner<N, VEC, 1, 5>(c, n, grads, mem, P);
+            if (N == 16 && n > 10 && n <= 12) return launch_learner<N, VEC, 1, 6>(c, n, grads, mem, P);
+            if (N == 16 && n > 12 && n <= 14) return launch_learner<N, VEC, 1, 7>(c, n, grads, mem, P);
+            return launch_learner<N, VEC, 1>(c, n, grads, mem, P);
         case 2: return launch_learner<N, VEC, LP_MID_T, 4, false, LP_MID_BLOCKS_PER_SM, LP_MID_EARLY>(c, n, grads, mem, P);
         // few learners: more blocks per SM and the first burst requested early
         case 4: return launch_learner<N, VEC, LP_FEW2_T, 2, false, LP_FEW2_BLOCKS_PER_SM, true>(c, n, grads, mem, P);

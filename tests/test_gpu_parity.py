@@ -33,6 +33,8 @@ def test_tiny_config_full(force_exact):
     (W.LARGE, 3_000_001, 5, 3),
     (W.RESNET50, 300_007, 20, 3),           # > 16 learners: second pointer-table size
     (W.RESNET50, 50_001, 130, 2),           # > 128 learners: third pointer-table size
+    (W.TINY, 300_007, 1, 3), (W.TINY, 300_007, 2, 3), (W.TINY, 300_007, 3, 4), (W.TINY, 300_007, 6, 3),   # every burst shape
+    (W.TINY, 300_007, 9, 2), (W.TINY, 300_007, 11, 2), (W.TINY, 300_007, 13, 2), (W.TINY, 300_007, 15, 2),
 ])
 def test_scaled_workloads(base, d, n, steps):
     _parity().workload_case(base.scaled(d, n=n), steps, DEV, want_path=0)
