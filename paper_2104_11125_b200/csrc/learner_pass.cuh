@@ -14,51 +14,19 @@
 
 namespace sc {
 
-#ifndef SC_LP_UNROLL
-#define SC_LP_UNROLL 8
-#endif
-#ifndef SC_LP_BLOCKS_PER_SM
-#define SC_LP_BLOCKS_PER_SM 2
-#endif
 constexpr int LP_THREADS = 256;            // x 4 coordinates = one tile
-constexpr int LP_UNROLL = SC_LP_UNROLL;    // learners in flight per thread
-constexpr int LP_BLOCKS_PER_SM = SC_LP_BLOCKS_PER_SM;
-#ifndef SC_ONE_T
-#define SC_ONE_T 2
-#endif
-#ifndef SC_ONE_BLOCKS
-#define SC_ONE_BLOCKS 4
-#endif
-#ifndef SC_FEW_T
-#define SC_FEW_T 2
-#endif
-#ifndef SC_FEW_BLOCKS
-#define SC_FEW_BLOCKS 4
-#endif
-#ifndef SC_FEW2_T
-#define SC_FEW2_T 1
-#endif
-#ifndef SC_FEW2_BLOCKS
-#define SC_FEW2_BLOCKS 5
-#endif
-constexpr int LP_ONE_T = SC_ONE_T;                 // tiles per burst of the single-learner form
-constexpr int LP_ONE_BLOCKS_PER_SM = SC_ONE_BLOCKS;
-constexpr int LP_FEW_T = SC_FEW_T;                 // tiles per burst with one learner
-constexpr int LP_FEW_BLOCKS_PER_SM = SC_FEW_BLOCKS;
-#ifndef SC_MID_T
-#define SC_MID_T 1
-#endif
-#ifndef SC_MID_BLOCKS
-#define SC_MID_BLOCKS 3
-#endif
-#ifndef SC_MID_EARLY
-#define SC_MID_EARLY 1
-#endif
-constexpr int LP_MID_T = SC_MID_T;                 // tiles per burst (of four learners) with 4 to 7 learners
-constexpr int LP_MID_BLOCKS_PER_SM = SC_MID_BLOCKS;
-constexpr bool LP_MID_EARLY = SC_MID_EARLY != 0;
-constexpr int LP_FEW2_T = SC_FEW2_T;               // tiles per burst (of two learners) with 2 or 3 learners
-constexpr int LP_FEW2_BLOCKS_PER_SM = SC_FEW2_BLOCKS;
+constexpr int LP_UNROLL = 8;               // pairs of 128-bit loads in flight per thread (tiles x learners of a burst)
+constexpr int LP_BLOCKS_PER_SM = 2;
+// burst shapes and blocks per SM by learner count (each measured against its neighbours on d = 25.6 M)
+constexpr int LP_ONE_T = 2;                // single-learner form (learner-per-GPU deployment): tiles per burst
+constexpr int LP_ONE_BLOCKS_PER_SM = 4;
+constexpr int LP_FEW_T = 2;                // one learner in scalecom_step
+constexpr int LP_FEW_BLOCKS_PER_SM = 4;
+constexpr int LP_FEW2_T = 1;               // 2 or 3 learners: bursts of two learners
+constexpr int LP_FEW2_BLOCKS_PER_SM = 5;
+constexpr int LP_MID_T = 1;                // 4 to 7 learners: bursts of four learners
+constexpr int LP_MID_BLOCKS_PER_SM = 3;
+constexpr bool LP_MID_EARLY = true;
 
 template <int N>
 struct PtrTable {
@@ -86,7 +54,12 @@ struct LearnerParams {
     float beta, omb, lr, nf;               // omb = 1 - beta rounded once in fp32; nf = (float)n
     const uint32_t* bitmap;                // [ntiles * 32]
     uint32_t* bitmap_clear;                // single-learner form: the same words, zeroed once read (or nullptr)
-    const uint32_t* tile_prefix;           // [ntiles + 1]
+    // ranks: either the exclusive prefix count of every tile ...
+    const uint32_t* tile_prefix;           // [ntiles + 1], used when tile_cnt is nullptr
+    // ... or the top-k selection kernel's count arrays (selected_before_tile)
+    const uint32_t* tile_cnt;              // [ntiles] or nullptr
+    const uint32_t* group_pre;             // [ngroups + 1]
+    uint32_t gshift;
     float* out_val;                        // [k]
     int32_t* out_idx;                      // [k]: the ascending index list, written here from the ranks
     float* gathered;                       // [n * k] or nullptr
@@ -133,7 +106,8 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
             const bool have = tile < P.ntiles;                         // uniform across the block
             pc[t] = have ? tile * TILE + tid * 4u : d;                 // d: nothing to do
             bw[t] = !have ? 0u : ONE ? P.bitmap[size_t(tile) * 32 + lane] : __ldg(&P.bitmap[size_t(tile) * 32 + lane]);
-            tp[t] = have ? __ldg(&P.tile_prefix[tile]) : 0u;
+            tp[t] = !have ? 0u : P.tile_cnt ? selected_before_tile(P.tile_cnt, P.group_pre, P.gshift, tile)
+                                            : __ldg(&P.tile_prefix[tile]);
         }
         float gv[LP_T][LP_L][4], mv[LP_T][LP_L][4];
         auto load_burst = [&](int i0) {

@@ -29,17 +29,21 @@ struct scalecom_ctx {
     void* ws = nullptr;
     size_t ws_bytes = 0;
     uint32_t *samp_hist = nullptr, *coarse_win = nullptr, *fine_hist = nullptr, *digit_hist = nullptr;
-    uint32_t *block_tot = nullptr, *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr, *leader_hint = nullptr;
+    uint32_t *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr, *leader_hint = nullptr;
+    uint32_t *tile_cnt = nullptr, *group_tot = nullptr, *group_pre = nullptr;   // the top-k selection's count arrays
+    uint32_t gshift = 5, ngroups = 1;
+    mutable uint32_t fine_parity = 0;  // which of the two fine histograms the next top-k launch counts in
     unsigned long long* barrier = nullptr;
     uint2* cand = nullptr;
     uint2* blist = nullptr;
-    uint32_t seg_cap = 0, ntiles = 0, tiles_per_block = 0;
+    uint32_t seg_cap = 0, ntiles = 0;
     size_t ctrl_region_bytes = 0;      // prefix of the workspace that reset() clears
 
     // launch geometry
     int sms = 0;
     uint32_t topk_blocks = 0, lp_blocks = 0;
     mutable bool select_fresh = false; // the bitmap and prefix counts are those of this handle's last scalecom_select
+    mutable bool select_counts = false; // ... and the ranks come from the count arrays (top-k selector), not tile_prefix
     mutable bool bitmap_zero = false;  // the bitmap holds no bits (scalecom_compress leaves it so; selection kernels do not)
     uint32_t samp_stride = 1, samp_target = 1;
 
@@ -105,10 +109,15 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 template <bool VEC>
-cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& P) {
+cudaError_t launch_topk(const scalecom_ctx* c, const TopkParams& params) {
     c->bitmap_zero = false;
     c->select_fresh = false;
-    void* args[] = {const_cast<TopkParams*>(&P)};
+    // two copies of the fine histogram used in turn: a launch counts in one and clears the other behind its stream
+    TopkParams P = params;
+    P.fine_hist = c->fine_hist + size_t(c->fine_parity) * NFINE;
+    P.fine_hist_next = c->fine_hist + size_t(c->fine_parity ^ 1u) * NFINE;
+    c->fine_parity ^= 1u;
+    void* args[] = {&P};
     return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&topk_select_kernel<VEC>), dim3(c->topk_blocks),
                                        dim3(TK_THREADS), args, sizeof(TopkShared), c->stream);
 }
@@ -239,6 +248,7 @@ cudaError_t launch_learner_n(const scalecom_ctx* c, int n, const float* const* g
 int init_workspace(scalecom_ctx* c) {
     c->bitmap_zero = false;
     c->select_fresh = false;
+    c->fine_parity = 0;
     if (cudaMemsetAsync(c->ws, 0, c->ctrl_region_bytes, c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     if (c->chunk_best && cudaMemsetAsync(c->chunk_best, 0, size_t(c->k) * 8, c->stream) != cudaSuccess)
         return SCALECOM_ERR_CUDA;
@@ -285,19 +295,21 @@ TopkParams make_topk_params(const scalecom_ctx* c, const float* g, const float* 
     tp.spin_limit = c->spin_limit;
     tp.samp_hist = c->samp_hist;
     tp.coarse_win = c->coarse_win;
-    tp.fine_hist = c->fine_hist;
+    tp.fine_hist = nullptr;        // set by launch_topk
+    tp.fine_hist_next = nullptr;
     tp.digit_hist = c->digit_hist;
-    tp.block_tot = c->block_tot;
     tp.ctrl = c->ctrl;
     tp.barrier = c->barrier;
     tp.cand = c->cand;
     tp.seg_cap = c->seg_cap;
     tp.blist = c->blist;
     tp.bitmap = c->bitmap;
-    tp.tile_prefix = c->tile_prefix;
+    tp.tile_cnt = c->tile_cnt;
+    tp.group_tot = c->group_tot;
+    tp.group_pre = c->group_pre;
     tp.ntiles = c->ntiles;
-    tp.tiles_per_block = c->tiles_per_block;
-    tp.out_idx = nullptr;          // the learner pass writes the index list from the ranks it computes anyway
+    tp.ngroups = c->ngroups;
+    tp.gshift = c->gshift;
     tp.spans = span_slot;
     return tp;
 }
@@ -330,6 +342,10 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     lp.nf = float(c->n);
     lp.bitmap = c->bitmap; lp.bitmap_clear = nullptr;
     lp.tile_prefix = c->tile_prefix;
+    const bool counts = c->selector == SCALECOM_SELECTOR_TOPK;     // that selector leaves counts, the others prefixes
+    lp.tile_cnt = counts ? c->tile_cnt : nullptr;
+    lp.group_pre = c->group_pre;
+    lp.gshift = c->gshift;
     lp.out_val = out_val;
     lp.out_idx = out_idx;
     lp.gathered = c->gathered;
@@ -434,7 +450,8 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->topk_blocks = uint32_t(c->sms * occ_topk);
     if (c->topk_blocks > chunks) c->topk_blocks = chunks;
     if (c->topk_blocks < 1) c->topk_blocks = 1;
-    c->tiles_per_block = (c->ntiles + c->topk_blocks - 1) / c->topk_blocks;
+    c->gshift = group_shift_for(c->ntiles);
+    c->ngroups = (c->ntiles + (1u << c->gshift) - 1u) >> c->gshift;
     c->lp_blocks = uint32_t(c->sms * occ_lp);
     if (c->lp_blocks > c->ntiles) c->lp_blocks = c->ntiles;
 
@@ -469,11 +486,12 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     size_t off = 0;
     auto carve = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
     const size_t o_samp = carve(NCOARSE * 4), o_cw = carve((WIN + 1) * 4), o_ctrl = carve(CT_WORDS * 4), o_bar = carve(256);
-    const size_t o_bt = carve(size_t(c->topk_blocks) * 4), o_lh = carve(size_t(n) * 4);
-    const size_t o_fine = carve(NFINE * 4), o_dh = carve(size_t(DH_PASSES) * DH_BINS * 4);
+    const size_t o_gt = carve(size_t(c->ngroups) * 4), o_lh = carve(size_t(n) * 4);
+    const size_t o_fine = carve(2 * size_t(NFINE) * 4), o_dh = carve(size_t(DH_PASSES) * DH_BINS * 4);
     c->ctrl_region_bytes = off;                 // everything the kernel expects to find zero
     const size_t o_cand = carve(size_t(c->seg_cap) * c->topk_blocks * TK_WARPS * 8), o_bl = carve(size_t(BCAP) * 8);
     const size_t o_bm = carve(size_t(c->ntiles) * 32 * 4), o_tp = carve((size_t(c->ntiles) + 1) * 4);
+    const size_t o_tc = carve(size_t(c->ntiles) * 4), o_gp = carve((size_t(c->ngroups) + 1) * 4);
     c->ws_bytes = off;
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -485,7 +503,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->coarse_win = reinterpret_cast<uint32_t*>(base + o_cw);
     c->ctrl = reinterpret_cast<uint32_t*>(base + o_ctrl);
     c->barrier = reinterpret_cast<unsigned long long*>(base + o_bar);
-    c->block_tot = reinterpret_cast<uint32_t*>(base + o_bt);
+    c->group_tot = reinterpret_cast<uint32_t*>(base + o_gt);
     c->leader_hint = reinterpret_cast<uint32_t*>(base + o_lh);
     c->fine_hist = reinterpret_cast<uint32_t*>(base + o_fine);
     c->digit_hist = reinterpret_cast<uint32_t*>(base + o_dh);
@@ -493,6 +511,8 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->blist = reinterpret_cast<uint2*>(base + o_bl);
     c->bitmap = reinterpret_cast<uint32_t*>(base + o_bm);
     c->tile_prefix = reinterpret_cast<uint32_t*>(base + o_tp);
+    c->tile_cnt = reinterpret_cast<uint32_t*>(base + o_tc);
+    c->group_pre = reinterpret_cast<uint32_t*>(base + o_gp);
 
     const bool ok = init_workspace(c) == SCALECOM_OK;
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) {
@@ -691,13 +711,22 @@ int scalecom_select(scalecom_ctx* c, const float* g, const float* m, int32_t* ou
         e = vec ? launch_layer_topk<true>(c, P) : launch_layer_topk<false>(c, P);
     } else {
         // one vector, one hint slot: the handle of a learner-per-GPU rank always sees the same learner
-        TopkParams tp = make_topk_params(c, g, m, c->leader_hint, true, nullptr);
-        tp.out_idx = out_idx;
+        const TopkParams tp = make_topk_params(c, g, m, c->leader_hint, true, nullptr);
         e = vec ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
+        if (e == cudaSuccess) {
+            // the ascending list from the bitmap and the counts the selection left
+            ++c->launches;
+            const uint32_t want = (c->ntiles + 7u) / 8u, cap = uint32_t(c->sms) * 8u;
+            emit_indices_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(c->bitmap, c->tile_cnt, c->group_pre, c->gshift,
+                                                                               c->ntiles, uint32_t(c->k), out_idx,
+                                                                               c->ctrl + CT_STATUS);
+            e = cudaGetLastError();
+        }
     }
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     c->select_fresh = true;
+    c->select_counts = c->selector == SCALECOM_SELECTOR_TOPK;
     return SCALECOM_OK;
 }
 
@@ -759,6 +788,8 @@ int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const i
     lp.n = 1;
     lp.beta = c->beta; lp.omb = 1.0f - c->beta; lp.lr = c->lr; lp.nf = 1.0f;
     lp.bitmap = c->bitmap; lp.bitmap_clear = c->bitmap; lp.tile_prefix = c->tile_prefix;
+    lp.tile_cnt = (!idx && c->select_counts) ? c->tile_cnt : nullptr;   // this handle's own top-k selection left counts
+    lp.group_pre = c->group_pre; lp.gshift = c->gshift;
     lp.out_val = out_gathered; lp.out_idx = c->scratch_idx;
     lp.gathered = nullptr; lp.weights = nullptr; lp.spans = nullptr;
     lp.status = c->ctrl + CT_STATUS;
