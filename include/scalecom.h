@@ -61,8 +61,10 @@ typedef enum scalecom_error {
  *   out    HOST, receives the handle.
  *   d      1 <= d <= 2^31 - 1.      n   1 <= n <= SCALECOM_MAX_LEARNERS.
  *   k      1 <= k <= d.             beta in (0, 1].   lr finite.
- * Allocates the scratch workspace (about d/8 + 24k + 1 MB bytes) on the current
- * device with cudaMalloc.  Errors: INVALID_ARG, NULL_PTR, ALLOC, CUDA.
+ * Allocates the scratch workspace on the current device with one cudaMalloc: about
+ * d/8 + d/128 + 48*k bytes + 0.4 MB (selection bitmap, per-tile counts, candidate
+ * segments, histograms); SCALECOM_Q_WORKSPACE_BYTES reports the exact figure.
+ * Errors: INVALID_ARG, NULL_PTR, ALLOC, CUDA.
  */
 int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float beta, float lr);
 
@@ -257,9 +259,11 @@ int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */
-#define SCALECOM_Q_PHASE_STAMP0     100 /* +i, i < 13: low 32 bits of the GPU nanosecond timer when block 0 of
-                                          the last top-k selection kernel reached phase boundary i (profiling
-                                          aid; boundaries 0-9 in phase order, 10-12 inside the final phase)    */
+#define SCALECOM_Q_PHASE_STAMP0     100 /* +i, i < 13: low 32 bits of the GPU nanosecond timer at phase boundary i of
+                                          the last top-k selection kernel (profiling aid): 0-7 as seen by block 0
+                                          (start; sample, barrier, bound; filter pass; barrier; k-th key located;
+                                          winners marked), 8-9 start and end of the completing work of the block
+                                          that finished last, 10-12 inside the marking phase of block 0        */
 int scalecom_query(scalecom_ctx* ctx, int item, int64_t* out);
 
 /*
@@ -279,10 +283,14 @@ int scalecom_kernel_ms(scalecom_ctx* ctx, float ms[3], int32_t* nsteps);
  * A process whose GPU memory is already fully owned by a framework's caching
  * allocator, or capped by a fixed partition, gets an error from cudaMalloc; a
  * latency-critical loop cannot afford the device-wide synchronisation cudaMalloc
- * implies.  Here the selection kernel's scratch is a fixed array inside the
- * library image (about 11 MB, present on every GPU that loads the library for
- * the life of the process), and the call performs no cudaMalloc, cudaFree or
- * any other allocating call.
+ * implies.  Here the selection kernels' scratch is a fixed array inside the
+ * library image (about 11 MB per GPU that uses this entry point, held until the
+ * process exits), and the call itself performs no cudaMalloc, cudaFree or any
+ * other allocating call.  The CUDA runtime places that array in device memory
+ * when the module is first used on a device, i.e. during the FIRST call on that
+ * device: make that call at start-up, before the rest of the application takes
+ * the GPU's memory (a first call made with no memory left fails with ALLOC) and
+ * before any stream capture begins.  Only the calls after it are allocation-free.
  *   g, m        DEVICE fp32[d]: the leader's gradient and memory; keys are |m + g|.
  *   d           1 <= d <= SCALECOM_STATIC_MAX_D (larger vectors: INVALID_ARG; use a handle).
  *   k           1 <= k <= d.
@@ -291,12 +299,12 @@ int scalecom_kernel_ms(scalecom_ctx* ctx, float ms[3], int32_t* nsteps);
  *               in-kernel wait expired, or 7 if a consistency check failed (out_idx is
  *               then undefined).
  *   cuda_stream cudaStream_t as void*; the work is asynchronous on it, on the current device.
- * The first call on each device looks up the array's device address and the
- * kernel's launch limits; make that first call before any stream capture begins.
+ * The first call on each device also looks up the array's device address and the
+ * kernels' launch limits.
  * All calls on a device share the one array, which still holds the previous
  * call's contents: each call clears what must start at zero, and two calls whose
  * GPU work overlaps (different streams, no dependency) race on it -- order them.
- * Errors: NULL_PTR, INVALID_ARG, ALIAS, CUDA.
+ * Errors: NULL_PTR, INVALID_ARG, ALIAS, ALLOC (first call on a device only), CUDA.
  */
 #define SCALECOM_STATIC_MAX_D (1 << 20)
 int scalecom_topk_static(const float* g, const float* m, int64_t d, int64_t k, int32_t* out_idx,

@@ -24,11 +24,6 @@ NVCC_FLAGS = [
 ]
 
 
-def _extra_flags():
-    """Extra nvcc flags for experiments (e.g. -DSC_TK_THREADS=1024); part of the build stamp."""
-    return os.environ.get("SCALECOM_NVCC_EXTRA", "").split()
-
-
 def _nvcc() -> str:
     exe = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     if not os.path.exists(exe):
@@ -37,7 +32,7 @@ def _nvcc() -> str:
 
 
 def source_hash() -> str:
-    h = hashlib.sha256(" ".join(NVCC_FLAGS + _extra_flags()).encode())
+    h = hashlib.sha256(" ".join(NVCC_FLAGS).encode())
     for name in SOURCES + HEADERS:
         with open(os.path.join(CSRC, name), "rb") as f:
             h.update(f.read())
@@ -58,7 +53,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and is_current():
         return LIB
     tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [_nvcc(), *NVCC_FLAGS, *_extra_flags(), *(["-Xptxas", "-v"] if verbose else []),
+    cmd = [_nvcc(), *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []),
            *[os.path.join(CSRC, s) for s in SOURCES], "-o", tmp]
     subprocess.run(cmd, check=True, cwd=HERE)
     os.replace(tmp, LIB)

@@ -17,23 +17,11 @@
 
 namespace sc {
 
-#ifndef SC_CS_THREADS
-#define SC_CS_THREADS 512
-#endif
-#ifndef SC_CS_BLOCKS_PER_SM
-#define SC_CS_BLOCKS_PER_SM 2
-#endif
-constexpr int CS_THREADS = SC_CS_THREADS;
-constexpr int CS_BLOCKS_PER_SM = SC_CS_BLOCKS_PER_SM;
-#ifndef SC_CS_GROUP
-#define SC_CS_GROUP 3
-#endif
-constexpr int CS_GROUP = SC_CS_GROUP;           // chunks a warp works on at a time
+constexpr int CS_THREADS = 512;
+constexpr int CS_BLOCKS_PER_SM = 2;
+constexpr int CS_GROUP = 3;                     // chunks a warp works on at a time
 constexpr int CS_UNROLL = 4;                    // rows of 32 coordinates of each of them in flight
-#ifndef SC_CS_RUN_GROUPS
-#define SC_CS_RUN_GROUPS 4
-#endif
-constexpr int CS_RUN = SC_CS_RUN_GROUPS * CS_GROUP;   // consecutive chunks a warp takes before moving on
+constexpr int CS_RUN = 4 * CS_GROUP;            // consecutive chunks a warp takes before moving on
 
 struct ChunkParams {
     const float* g;

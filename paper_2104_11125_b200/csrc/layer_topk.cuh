@@ -26,16 +26,10 @@
 
 namespace sc {
 
-#ifndef SC_LT_BLOCKS_PER_SM
-#define SC_LT_BLOCKS_PER_SM 2
-#endif
-#ifndef SC_LT_UNROLL
-#define SC_LT_UNROLL 2
-#endif
 constexpr int LT_THREADS = 512;
 constexpr int LT_WARPS = LT_THREADS / 32;
-constexpr int LT_BLOCKS_PER_SM = SC_LT_BLOCKS_PER_SM;
-constexpr int LT_UNROLL = SC_LT_UNROLL;             // spans whose loads a thread has in flight
+constexpr int LT_BLOCKS_PER_SM = 2;
+constexpr int LT_UNROLL = 2;             // spans whose loads a thread has in flight
 constexpr uint32_t LT_SPAN = LT_THREADS * 4;        // coordinates a block takes per iteration (two tiles)
 constexpr uint32_t LT_BINS = 2048;                  // widest digit: 11 bits
 // Per-layer marker in shared memory (S.w): the key rounds are still running / the layer is done (keep every

@@ -135,14 +135,18 @@ cudaError_t launch_chunk(const scalecom_ctx* c, const ChunkParams& P) {
 // Scratch of the per-layer exact selector, made at the first launch after the layers were set.
 int ensure_layer_ws(scalecom_ctx* c) {
     if (c->lt_ws) return SCALECOM_OK;
-    int occ = 0;
+    int occ = 0, occ_unaligned = 0;
     if (cudaFuncSetAttribute(layer_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(sizeof(LayerTopkShared))) != cudaSuccess ||
         cudaFuncSetAttribute(layer_topk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              int(sizeof(LayerTopkShared))) != cudaSuccess ||
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, layer_topk_kernel<true>, LT_THREADS, sizeof(LayerTopkShared)) !=
-            cudaSuccess || occ < 1)
+            cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_unaligned, layer_topk_kernel<false>, LT_THREADS,
+                                                      sizeof(LayerTopkShared)) != cudaSuccess)
         return SCALECOM_ERR_CUDA;
+    if (occ_unaligned < occ) occ = occ_unaligned;          // one grid serves both instantiations of the cooperative kernel
+    if (occ < 1) return SCALECOM_ERR_CUDA;
     if (occ > LT_BLOCKS_PER_SM) occ = LT_BLOCKS_PER_SM;
     c->lt_blocks = uint32_t(c->sms * occ);
     const size_t nl = c->nlayers;
@@ -292,6 +296,8 @@ TopkParams make_topk_params(const scalecom_ctx* c, const float* g, const float* 
     tp.force_exact = c->force_exact;
     tp.use_hint = use_hint ? c->use_hint : 0u;
     tp.leader_hint = leader_hint;
+    tp.all_hints = leader_hint ? c->leader_hint : nullptr;
+    tp.n_hints = uint32_t(c->n);
     tp.spin_limit = c->spin_limit;
     tp.samp_hist = c->samp_hist;
     tp.coarse_win = c->coarse_win;
@@ -536,11 +542,11 @@ int scalecom_step(scalecom_ctx* c, const float* const* grads, float* const* mem,
 
 int scalecom_step_host(scalecom_ctx* c, const float* const* host_grads, float* const* mem, float* weights, int64_t t,
                        int32_t* host_idx, float* host_val) {
-    if (!c || !host_grads || !mem || !host_idx || !host_val) return SCALECOM_ERR_NULL_PTR;
-    if (t < 0) return SCALECOM_ERR_INVALID_ARG;
-    if (c->poisoned) return SCALECOM_ERR_BAD_STATE;
-    for (int i = 0; i < c->n; ++i)
-        if (!host_grads[i] || !mem[i]) return SCALECOM_ERR_NULL_PTR;
+    // every argument is checked before anything is allocated, copied or launched (host and device pointers share
+    // one address space, so the distinctness checks of scalecom_step apply as they are)
+    int rc = check_step_args(c, reinterpret_cast<const void* const*>(host_grads), reinterpret_cast<const void* const*>(mem),
+                             weights, t, host_idx, host_val);
+    if (rc != SCALECOM_OK) return rc;
     DeviceGuard guard(c->device);
     if (!guard.ok) return SCALECOM_ERR_CUDA;
     if (!c->stage_g) {
@@ -555,18 +561,12 @@ int scalecom_step_host(scalecom_ctx* c, const float* const* host_grads, float* c
         }
     }
     const float* dev_g[SCALECOM_MAX_LEARNERS];
-    const int leader = int(t % c->n);
-    // the leader's gradient goes first: the selection kernel needs nothing else
-    for (int j = 0; j < c->n; ++j) {
-        const int i = (leader + j) % c->n;
+    for (int i = 0; i < c->n; ++i) {
         float* dst = c->stage_g + size_t(i) * size_t(c->d);
         dev_g[i] = dst;
         if (cudaMemcpyAsync(dst, host_grads[i], size_t(c->d) * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
             return SCALECOM_ERR_CUDA;
     }
-    int rc = check_step_args(c, reinterpret_cast<const void* const*>(dev_g), reinterpret_cast<const void* const*>(mem),
-                             weights, t, c->stage_idx, c->stage_val);
-    if (rc != SCALECOM_OK) return rc;
     rc = do_step(c, dev_g, mem, weights, t, c->stage_idx, c->stage_val);
     if (rc != SCALECOM_OK) return rc;
     if (cudaMemcpyAsync(host_idx, c->stage_idx, size_t(c->k) * 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
@@ -885,9 +885,18 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
             if (value == SCALECOM_SELECTOR_CHUNK && !c->chunk_best) {
                 DeviceGuard guard(c->device);
                 int occ = 0;
-                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, chunk_select_kernel<true, true>, CS_THREADS, 0) != cudaSuccess ||
-                    occ < 1)
-                    return SCALECOM_ERR_CUDA;
+                // the smallest occupancy of the four instantiations: one grid serves them all
+                {
+                    int o[4] = {0, 0, 0, 0};
+                    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[0], chunk_select_kernel<true, true>, CS_THREADS, 0) != cudaSuccess ||
+                        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[1], chunk_select_kernel<true, false>, CS_THREADS, 0) != cudaSuccess ||
+                        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[2], chunk_select_kernel<false, true>, CS_THREADS, 0) != cudaSuccess ||
+                        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o[3], chunk_select_kernel<false, false>, CS_THREADS, 0) != cudaSuccess)
+                        return SCALECOM_ERR_CUDA;
+                    occ = o[0];
+                    for (int q = 1; q < 4; ++q) occ = o[q] < occ ? o[q] : occ;
+                    if (occ < 1) return SCALECOM_ERR_CUDA;
+                }
                 if (occ > CS_BLOCKS_PER_SM) occ = CS_BLOCKS_PER_SM;
                 const int64_t per_block = int64_t(CS_THREADS / 32) * CS_RUN;                   // chunks one block takes per round
                 const uint32_t need = uint32_t((c->k + per_block - 1) / per_block);

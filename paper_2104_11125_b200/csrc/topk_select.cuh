@@ -93,6 +93,8 @@ struct TopkParams {
     uint32_t force_exact;
     uint32_t use_hint;         // 1: start from the bound earlier launches left behind
     uint32_t* leader_hint;     // this leader's own entry (bin + 1 of its last threshold, 0 = none), or nullptr
+    uint32_t* all_hints;       // every leader's entry [n_hints] (or nullptr): forgotten when a hint turns out useless
+    uint32_t n_hints;
     uint32_t spin_limit;
     // the histograms, group_tot and the counters in ctrl are all zero on entry and all zero again on exit
     uint32_t* samp_hist;       // [NCOARSE]
@@ -822,8 +824,15 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
             // the threshold: late in a run one bin holds about k of them)
             if (hint && !used_hint) P.ctrl[CT_MARGIN] = hint_overflowed ? 0u : 1u;
             else if (used_hint && M > 3u * k) P.ctrl[CT_MARGIN] = 0u;
+            // a useless hint means the scale moved under every learner: what the other leaders remember (and the
+            // change this one is about to record against its own stale value) would mislead the next steps, which
+            // start from this step's bin instead until each leader has led again
+            const bool forget = hint && !used_hint && P.all_hints;
+            if (forget)
+                for (uint32_t i = 0; i < P.n_hints; ++i) P.all_hints[i] = 0u;
             const uint32_t cbk = st.nbits >= 13 ? uint32_t(st.prefix >> (st.nbits - 13)) : 0u;
-            if (cbk && own_prev) P.ctrl[CT_DRIFT] = uint32_t(int32_t(cbk) - int32_t(own_prev - 1u));
+            if (forget) P.ctrl[CT_DRIFT] = 0u;
+            else if (cbk && own_prev) P.ctrl[CT_DRIFT] = uint32_t(int32_t(cbk) - int32_t(own_prev - 1u));
             P.ctrl[CT_HINT] = cbk ? cbk + 1u : 0u;
             if (P.leader_hint) *P.leader_hint = cbk ? cbk + 1u : 0u;
         }

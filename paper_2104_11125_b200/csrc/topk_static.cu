@@ -42,7 +42,7 @@ constexpr size_t OFF_CAND = OFF_BL + al(size_t(BCAP) * 8);
 constexpr size_t CAND_ENTRIES = size_t(MAX_D) + 32u * MAX_BLOCKS * TK_WARPS;   // every warp's share of the vector + slack
 constexpr size_t SCRATCH_BYTES = OFF_CAND + al(CAND_ENTRIES * 8);
 
-// About 11 MB, held by every GPU that loads the library until the process exits.
+// About 11 MB, held by every GPU on which this entry point has been called, until the process exits.
 // In host code this name is only a stand-in for the symbol, never a device
 // address: the address the kernel gets comes from cudaGetSymbolAddress below.
 static __device__ __align__(256) unsigned char g_scratch[SCRATCH_BYTES];
@@ -56,8 +56,11 @@ DeviceSetup g_setup[MAX_DEVICES];
 std::mutex g_mu;
 
 int setup_device(int dev, DeviceSetup& su) {
+    // (with lazy module loading this is also where the runtime places the array in device memory)
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_scratch) != cudaSuccess || !p) return SCALECOM_ERR_CUDA;
+    const cudaError_t es = cudaGetSymbolAddress(&p, g_scratch);
+    if (es == cudaErrorMemoryAllocation) return SCALECOM_ERR_ALLOC;
+    if (es != cudaSuccess || !p) return SCALECOM_ERR_CUDA;
     int sms = 0, coop = 0, occ = 0, o2 = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop ||
@@ -126,6 +129,8 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
     P.force_exact = 0;
     P.use_hint = 0;               // the scratch is shared by unrelated callers: no carry-over between calls
     P.leader_hint = nullptr;
+    P.all_hints = nullptr;
+    P.n_hints = 0;
     P.spin_limit = 1u << 22;
     P.samp_hist = reinterpret_cast<uint32_t*>(base + OFF_SAMP);
     P.coarse_win = reinterpret_cast<uint32_t*>(base + OFF_CW);

@@ -24,7 +24,7 @@ def _windows(d):
     return [(0, WIN), (mid, mid + WIN), (d - WIN - 3, d)]
 
 
-def fullsize_case(w, steps=2):
+def fullsize_case(w, steps=2, strict_paths=True):
     import paper_2104_11125_b200 as sc
     from paper_2104_11125_b200 import binding
     from tests.parity import rel_err, REL_TOL
@@ -41,6 +41,7 @@ def fullsize_case(w, steps=2):
     m_full = {i: np.zeros(d, np.float32) for i in leaders}
     m_win = [[np.zeros(b - a, np.float32) for (a, b) in wins] for _ in range(n)]
     th_win = [th0[a:b].copy() for (a, b) in wins]
+    paths = []
     with sc.Context(d, n, k, w.beta, w.lr) as ctx:
         ctx.set_gathered(G)
         for t in range(steps):
@@ -48,7 +49,9 @@ def fullsize_case(w, steps=2):
             ctx.step(g, m_g, th_g, t, idx, val)
             assert ctx.status() == 0
             path = ctx.query(binding.Q_LAST_TOPK_PATH)
-            assert path == (binding.PATH_SAMPLED if t == 0 else binding.PATH_HINTED), "step %d took path %d" % (t, path)
+            paths.append(path)
+            if strict_paths:
+                assert path == (binding.PATH_SAMPLED if t == 0 else binding.PATH_HINTED), "step %d took path %d" % (t, path)
             L = t % n
             # ---- selection: full, bit-exact ----
             acc = oracle.accumulate(g[L].cpu().numpy(), m_full[L])
@@ -85,6 +88,7 @@ def fullsize_case(w, steps=2):
                 thw = th_g[a:b].cpu().numpy()
                 assert rel_err(thw, th_win[wi]) <= REL_TOL and np.array_equal(thw, th_win[wi])
             del g
+    return paths
 
 
 def test_config2_resnet50_full_oracle_step():
@@ -101,7 +105,7 @@ def test_config3_transformer_windows():
     fullsize_case(W.TRANSFORMER, steps=2)
 
 
-@pytest.mark.parametrize("n", [32, 128])
+@pytest.mark.parametrize("n", [32, 64, 128])
 def test_config4_learner_sweep_windows(n):
     fullsize_case(W.sweep(n), steps=2)
 
