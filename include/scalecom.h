@@ -195,6 +195,16 @@ int scalecom_compress(scalecom_ctx* ctx, const float* g, float* m, const int32_t
  */
 int scalecom_compress_scatter(scalecom_ctx* ctx, const float* g, float* m, const int32_t* idx, float* out_gathered,
                               float* const* dst, int32_t n_dst, uint32_t* const* flag_dst, uint32_t tag);
+
+/*
+ * Give the handle's device access to the memory of another device of this process (cudaDeviceEnablePeerAccess
+ * with the handle's device current), which the stores of scalecom_compress_scatter into a peer's rows and the
+ * polls of scalecom_reduce_rows need when the rows live on another GPU (the exchange of the kept values in the
+ * paper's deployment, Section 4 / Appendix E).  peer_device is a device ordinal of this process.  Already enabled
+ * counts as success; the handle's own device is accepted and does nothing.
+ * Errors: NULL_PTR, INVALID_ARG (no such device, or the hardware offers no peer access between the two), CUDA.
+ */
+int scalecom_enable_peer_access(scalecom_ctx* ctx, int32_t peer_device);
 int scalecom_reduce_rows(scalecom_ctx* ctx, const float* rows, int32_t n_rows, float* out_val, const int32_t* idx,
                          float* weights, const uint32_t* wait_flags, uint32_t tag);
 

@@ -30,18 +30,19 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cltk_oracle.c")
 _INC = os.path.join(_HERE, "cltk_oracle_body.inc")
+_SRC_MT = os.path.join(_HERE, "cltk_oracle_mt.c")
 _LIB = os.path.join(_HERE, "libcltk_oracle.so")
 
-CFLAGS = ["-std=c99", "-O2", "-ffp-contract=off", "-fPIC", "-shared"]
+CFLAGS = ["-std=c99", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-pthread"]
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc if the shared object is missing or stale."""
     stale = (not os.path.exists(_LIB)
-             or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_INC)))
+             or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_INC), os.path.getmtime(_SRC_MT)))
     if force or stale:
         tmp = _LIB + ".tmp.%d" % os.getpid()
-        subprocess.run(["gcc", *CFLAGS, _SRC, "-o", tmp, "-lm"], check=True, cwd=_HERE)
+        subprocess.run(["gcc", *CFLAGS, _SRC, _SRC_MT, "-o", tmp, "-lm"], check=True, cwd=_HERE)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -77,7 +78,17 @@ def _load():
             f = getattr(_lib, "oracle_apply_" + sfx); f.restype = None; f.argtypes = [vp, vp, vp, i64, real]
             f = getattr(_lib, "oracle_step_" + sfx); f.restype = ctypes.c_int
             f.argtypes = [vp, vp, vp, i64, i32, i64, i64, real, real, vp, vp, vp]
+        f = _lib.oracle_step_threads_f32; f.restype = ctypes.c_int
+        f.argtypes = [vp, vp, vp, i64, i32, i64, i64, ctypes.c_float, ctypes.c_float, i32, vp, vp, vp]
     return _lib
+
+
+def host_cores() -> int:
+    """Host cores this process may run on."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:  # pragma: no cover
+        return os.cpu_count() or 1
 
 
 def _sfx(dtype) -> str:
@@ -223,9 +234,10 @@ def apply(theta: np.ndarray, idx: np.ndarray, val: np.ndarray, lr: float) -> Non
 
 
 def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: bool = True,
-         selector: str = "topk", layers=None):
+         selector: str = "topk", layers=None, threads: int = 1):
     """One iteration of Algorithm 1 ("topk": Eq. 2 on the leader; "chunk": chunk-wise selection,
-    with per-layer rates when layers = (sizes, keep) is given).
+    with per-layer rates when layers = (sizes, keep) is given).  threads > 1 (fp32, "topk", no layers):
+    the same routines with their loops spread over that many threads -- identical results, shorter wall clock.
 
     g, m: lists of n ndarrays of d values (m updated in place); theta: ndarray
     of d values updated in place, or None.  Returns (idx, val, G) with G the
@@ -251,6 +263,16 @@ def step(g, m, theta, t: int, k: int, beta: float, lr: float, want_gathered: boo
         nl, szp, kpp = sz.size, _p(sz), _p(kp)
     else:
         nl, szp, kpp = 0, None, None
+    if threads > 1:
+        if np.dtype(dtype) != np.float32 or selector != "topk" or layers is not None:
+            raise ValueError("the threaded step is fp32, exact top-k, no layers")
+        rc = lib.oracle_step_threads_f32(
+            ctypes.cast(gp, ctypes.c_void_p), ctypes.cast(mp, ctypes.c_void_p),
+            _p(theta) if theta is not None else None, int(t), n, d, int(k), float(beta), float(lr), int(threads),
+            _p(idx), _p(val), _p(G) if G is not None else None)
+        if rc != 0:
+            raise MemoryError("oracle_step_threads")
+        return idx, val, G
     rc = getattr(lib, "oracle_step_layers_" + _sfx(dtype))(
         ctypes.cast(gp, ctypes.c_void_p), ctypes.cast(mp, ctypes.c_void_p),
         _p(theta) if theta is not None else None,

@@ -31,7 +31,7 @@ EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",
     "scalecom_set_gathered", "scalecom_apply_update", "scalecom_status", "scalecom_reset",
     "scalecom_set_option", "scalecom_query", "scalecom_kernel_ms", "scalecom_strerror",
-    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_overlap", "scalecom_cosine_distance", "scalecom_set_layers", "scalecom_select", "scalecom_compress", "scalecom_reduce_rows", "scalecom_compress_scatter",
+    "scalecom_topk_static", "scalecom_kernel_span_ms", "scalecom_enable_peer_access", "scalecom_overlap", "scalecom_cosine_distance", "scalecom_set_layers", "scalecom_select", "scalecom_compress", "scalecom_reduce_rows", "scalecom_compress_scatter",
 )
 STATIC_MAX_D = 1 << 20
 
@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
         L.scalecom_compress_scatter.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, ctypes.c_uint32]
         L.scalecom_reduce_rows.restype = ctypes.c_int
         L.scalecom_reduce_rows.argtypes = [vp, vp, i32, vp, vp, vp, vp, ctypes.c_uint32]
+        L.scalecom_enable_peer_access.restype = ctypes.c_int
+        L.scalecom_enable_peer_access.argtypes = [vp, i32]
         L.scalecom_strerror.restype = ctypes.c_char_p
         L.scalecom_strerror.argtypes = [ctypes.c_int]
         _lib = L
@@ -195,6 +197,10 @@ class Context:
         ptr = None if buf is None else _dev_f32(buf, self.n * self.k, "gathered")
         _check(lib().scalecom_set_gathered(self._h, ptr), "scalecom_set_gathered")
         self._gathered = buf
+
+    def enable_peer_access(self, peer_device: int) -> None:
+        """Let this handle's device store into (and load from) memory of another device of the process."""
+        _check(lib().scalecom_enable_peer_access(self._h, int(peer_device)), "scalecom_enable_peer_access")
 
     def set_option(self, option: int, value: int) -> None:
         _check(lib().scalecom_set_option(self._h, option, int(value)), "scalecom_set_option")
@@ -306,6 +312,28 @@ class Context:
             raise TypeError("out_idx must be a contiguous CUDA int32 tensor of k elements")
         _check(scalecom_step(self._h, gp, mp, wp, t, out_idx.data_ptr(), _dev_f32(out_val, self.k, "out_val")),
                "scalecom_step")
+
+    def prepare_step(self, grad_batches: Sequence[Sequence[torch.Tensor]], mem: Sequence[torch.Tensor],
+                     weights: Optional[torch.Tensor], out_idx: torch.Tensor, out_val: torch.Tensor):
+        """Marshal the arguments of scalecom_step once for callers that step many times over the same buffers:
+        returns call(b, t) = scalecom_step with gradient set grad_batches[b] at iteration t.  The tensors must stay
+        alive and in place for as long as the callable is used."""
+        if len(mem) != self.n or any(len(g) != self.n for g in grad_batches):
+            raise ValueError("expected %d gradient and %d memory tensors" % (self.n, self.n))
+        tables = [_ptr_array([_dev_f32(g, self.d, "grads[%d]" % i) for i, g in enumerate(gs)]) for gs in grad_batches]
+        mtab = _ptr_array([_dev_f32(m, self.d, "mem[%d]" % i) for i, m in enumerate(mem)])
+        gp = [ctypes.cast(tb, ctypes.c_void_p) for tb in tables]
+        mp = ctypes.cast(mtab, ctypes.c_void_p)
+        wp = None if weights is None else _dev_f32(weights, self.d, "weights")
+        ip, vp = self._idx(out_idx), _dev_f32(out_val, self.k, "out_val")
+        fn, h = lib().scalecom_step, self._h
+        keep = (tables, mtab, grad_batches, mem, weights, out_idx, out_val)
+
+        def call(b: int, t: int, _keep=keep) -> None:
+            rc = fn(h, gp[b], mp, wp, t, ip, vp)
+            if rc != OK:
+                raise ScaleComError(rc, "scalecom_step")
+        return call
 
     def step_host(self, host_grads: Sequence[torch.Tensor], mem: Sequence[torch.Tensor],
                   weights: Optional[torch.Tensor], t: int, host_idx: torch.Tensor, host_val: torch.Tensor) -> None:

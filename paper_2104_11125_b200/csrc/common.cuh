@@ -68,19 +68,6 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
 
 __device__ __forceinline__ uint32_t warp_sum(uint32_t v) { return __reduce_add_sync(FULL, v); }
 
-// ---- ranks from the selection kernel's count arrays ---------------------------------------------------
-// Number of selected coordinates before tile `tile` in the ascending index list: the exclusive prefix at the
-// start of the tile's group (2^gshift consecutive tiles) plus the counts of the group's earlier tiles.  Called
-// by a whole warp; every lane returns the result.
-__device__ __forceinline__ uint32_t selected_before_tile(const uint32_t* __restrict__ tile_cnt,
-                                                         const uint32_t* __restrict__ group_pre, uint32_t gshift,
-                                                         uint32_t tile) {
-    const uint32_t grp = tile >> gshift;
-    uint32_t sum = 0;
-    for (uint32_t j = (grp << gshift) + lane_id(); j < tile; j += 32u) sum += __ldg(tile_cnt + j);
-    return warp_sum(sum) + __ldg(group_pre + grp);
-}
-
 // ---- in-kernel time spans ------------------------------------------------------------------------
 // A kernel given a non-null `sp` accumulates {~(earliest block start), latest block end} on the
 // nanosecond global timer into sp[0], sp[1] (both with atomicMax on zero-initialised words), which

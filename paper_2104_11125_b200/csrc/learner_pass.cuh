@@ -54,12 +54,7 @@ struct LearnerParams {
     float beta, omb, lr, nf;               // omb = 1 - beta rounded once in fp32; nf = (float)n
     const uint32_t* bitmap;                // [ntiles * 32]
     uint32_t* bitmap_clear;                // single-learner form: the same words, zeroed once read (or nullptr)
-    // ranks: either the exclusive prefix count of every tile ...
-    const uint32_t* tile_prefix;           // [ntiles + 1], used when tile_cnt is nullptr
-    // ... or the top-k selection kernel's count arrays (selected_before_tile)
-    const uint32_t* tile_cnt;              // [ntiles] or nullptr
-    const uint32_t* group_pre;             // [ngroups + 1]
-    uint32_t gshift;
+    const uint32_t* tile_prefix;           // [ntiles + 1]
     float* out_val;                        // [k]
     int32_t* out_idx;                      // [k]: the ascending index list, written here from the ranks
     float* gathered;                       // [n * k] or nullptr
@@ -106,8 +101,7 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
             const bool have = tile < P.ntiles;                         // uniform across the block
             pc[t] = have ? tile * TILE + tid * 4u : d;                 // d: nothing to do
             bw[t] = !have ? 0u : ONE ? P.bitmap[size_t(tile) * 32 + lane] : __ldg(&P.bitmap[size_t(tile) * 32 + lane]);
-            tp[t] = !have ? 0u : P.tile_cnt ? selected_before_tile(P.tile_cnt, P.group_pre, P.gshift, tile)
-                                            : __ldg(&P.tile_prefix[tile]);
+            tp[t] = have ? __ldg(&P.tile_prefix[tile]) : 0u;
         }
         float gv[LP_T][LP_L][4], mv[LP_T][LP_L][4];
         auto load_burst = [&](int i0) {

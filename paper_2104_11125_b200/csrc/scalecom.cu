@@ -30,8 +30,8 @@ struct scalecom_ctx {
     size_t ws_bytes = 0;
     uint32_t *samp_hist = nullptr, *coarse_win = nullptr, *fine_hist = nullptr, *digit_hist = nullptr;
     uint32_t *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr, *leader_hint = nullptr;
-    uint32_t *tile_cnt = nullptr, *group_tot = nullptr, *group_pre = nullptr;   // the top-k selection's count arrays
-    uint32_t gshift = 5, ngroups = 1;
+    uint32_t *block_tot = nullptr;
+    uint32_t tiles_per_block = 0;
     mutable uint32_t fine_parity = 0;  // which of the two fine histograms the next top-k launch counts in
     unsigned long long* barrier = nullptr;
     uint2* cand = nullptr;
@@ -43,7 +43,6 @@ struct scalecom_ctx {
     int sms = 0;
     uint32_t topk_blocks = 0, lp_blocks = 0;
     mutable bool select_fresh = false; // the bitmap and prefix counts are those of this handle's last scalecom_select
-    mutable bool select_counts = false; // ... and the ranks come from the count arrays (top-k selector), not tile_prefix
     mutable bool bitmap_zero = false;  // the bitmap holds no bits (scalecom_compress leaves it so; selection kernels do not)
     uint32_t samp_stride = 1, samp_target = 1;
 
@@ -310,12 +309,11 @@ TopkParams make_topk_params(const scalecom_ctx* c, const float* g, const float* 
     tp.seg_cap = c->seg_cap;
     tp.blist = c->blist;
     tp.bitmap = c->bitmap;
-    tp.tile_cnt = c->tile_cnt;
-    tp.group_tot = c->group_tot;
-    tp.group_pre = c->group_pre;
+    tp.tile_prefix = c->tile_prefix;
+    tp.block_tot = c->block_tot;
     tp.ntiles = c->ntiles;
-    tp.ngroups = c->ngroups;
-    tp.gshift = c->gshift;
+    tp.tiles_per_block = c->tiles_per_block;
+    tp.out_idx = nullptr;          // (scalecom_select asks for the list; a step's learner pass writes it from its ranks)
     tp.spans = span_slot;
     return tp;
 }
@@ -348,10 +346,6 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     lp.nf = float(c->n);
     lp.bitmap = c->bitmap; lp.bitmap_clear = nullptr;
     lp.tile_prefix = c->tile_prefix;
-    const bool counts = c->selector == SCALECOM_SELECTOR_TOPK;     // that selector leaves counts, the others prefixes
-    lp.tile_cnt = counts ? c->tile_cnt : nullptr;
-    lp.group_pre = c->group_pre;
-    lp.gshift = c->gshift;
     lp.out_val = out_val;
     lp.out_idx = out_idx;
     lp.gathered = c->gathered;
@@ -430,17 +424,16 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     cudaError_t e = cudaGetDevice(&c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(topk_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(TopkShared)));
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(topk_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(TopkShared)));
-    if (e == cudaSuccess)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_topk, topk_select_kernel<true>, TK_THREADS, sizeof(TopkShared));
-    if (e == cudaSuccess) {
-        int o2 = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o2, topk_select_kernel<false>, TK_THREADS, sizeof(TopkShared));
-        if (o2 < occ_topk) occ_topk = o2;
-    }
+    // one grid serves both instantiations of the cooperative selection kernel: the smaller occupancy counts
+    occ_topk = 1 << 20;
+    auto prepare = [&](auto kernel) {
+        int o = 0;
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(TopkShared)));
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kernel, TK_THREADS, sizeof(TopkShared));
+        if (o < occ_topk) occ_topk = o;
+    };
+    prepare(topk_select_kernel<true>);
+    prepare(topk_select_kernel<false>);
     if (e == cudaSuccess)
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_lp, learner_pass_kernel<16, true, 1, LP_UNROLL>, LP_THREADS, 0);
     if (e != cudaSuccess || !coop || occ_topk < 1 || occ_lp < 1) {
@@ -456,8 +449,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->topk_blocks = uint32_t(c->sms * occ_topk);
     if (c->topk_blocks > chunks) c->topk_blocks = chunks;
     if (c->topk_blocks < 1) c->topk_blocks = 1;
-    c->gshift = group_shift_for(c->ntiles);
-    c->ngroups = (c->ntiles + (1u << c->gshift) - 1u) >> c->gshift;
+    c->tiles_per_block = (c->ntiles + c->topk_blocks - 1) / c->topk_blocks;
     c->lp_blocks = uint32_t(c->sms * occ_lp);
     if (c->lp_blocks > c->ntiles) c->lp_blocks = c->ntiles;
 
@@ -492,12 +484,11 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     size_t off = 0;
     auto carve = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
     const size_t o_samp = carve(NCOARSE * 4), o_cw = carve((WIN + 1) * 4), o_ctrl = carve(CT_WORDS * 4), o_bar = carve(256);
-    const size_t o_gt = carve(size_t(c->ngroups) * 4), o_lh = carve(size_t(n) * 4);
+    const size_t o_lh = carve(size_t(n) * 4), o_bt = carve(size_t(c->topk_blocks) * 4);
     const size_t o_fine = carve(2 * size_t(NFINE) * 4), o_dh = carve(size_t(DH_PASSES) * DH_BINS * 4);
     c->ctrl_region_bytes = off;                 // everything the kernel expects to find zero
     const size_t o_cand = carve(size_t(c->seg_cap) * c->topk_blocks * TK_WARPS * 8), o_bl = carve(size_t(BCAP) * 8);
     const size_t o_bm = carve(size_t(c->ntiles) * 32 * 4), o_tp = carve((size_t(c->ntiles) + 1) * 4);
-    const size_t o_tc = carve(size_t(c->ntiles) * 4), o_gp = carve((size_t(c->ngroups) + 1) * 4);
     c->ws_bytes = off;
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -509,7 +500,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->coarse_win = reinterpret_cast<uint32_t*>(base + o_cw);
     c->ctrl = reinterpret_cast<uint32_t*>(base + o_ctrl);
     c->barrier = reinterpret_cast<unsigned long long*>(base + o_bar);
-    c->group_tot = reinterpret_cast<uint32_t*>(base + o_gt);
+    c->block_tot = reinterpret_cast<uint32_t*>(base + o_bt);
     c->leader_hint = reinterpret_cast<uint32_t*>(base + o_lh);
     c->fine_hist = reinterpret_cast<uint32_t*>(base + o_fine);
     c->digit_hist = reinterpret_cast<uint32_t*>(base + o_dh);
@@ -517,8 +508,6 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->blist = reinterpret_cast<uint2*>(base + o_bl);
     c->bitmap = reinterpret_cast<uint32_t*>(base + o_bm);
     c->tile_prefix = reinterpret_cast<uint32_t*>(base + o_tp);
-    c->tile_cnt = reinterpret_cast<uint32_t*>(base + o_tc);
-    c->group_pre = reinterpret_cast<uint32_t*>(base + o_gp);
 
     const bool ok = init_workspace(c) == SCALECOM_OK;
     if (!ok || cudaStreamSynchronize(c->stream) != cudaSuccess) {
@@ -711,22 +700,13 @@ int scalecom_select(scalecom_ctx* c, const float* g, const float* m, int32_t* ou
         e = vec ? launch_layer_topk<true>(c, P) : launch_layer_topk<false>(c, P);
     } else {
         // one vector, one hint slot: the handle of a learner-per-GPU rank always sees the same learner
-        const TopkParams tp = make_topk_params(c, g, m, c->leader_hint, true, nullptr);
+        TopkParams tp = make_topk_params(c, g, m, c->leader_hint, true, nullptr);
+        tp.out_idx = out_idx;
         e = vec ? launch_topk<true>(c, tp) : launch_topk<false>(c, tp);
-        if (e == cudaSuccess) {
-            // the ascending list from the bitmap and the counts the selection left
-            ++c->launches;
-            const uint32_t want = (c->ntiles + 7u) / 8u, cap = uint32_t(c->sms) * 8u;
-            emit_indices_kernel<<<want < cap ? want : cap, 256, 0, c->stream>>>(c->bitmap, c->tile_cnt, c->group_pre, c->gshift,
-                                                                               c->ntiles, uint32_t(c->k), out_idx,
-                                                                               c->ctrl + CT_STATUS);
-            e = cudaGetLastError();
-        }
     }
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
     c->select_fresh = true;
-    c->select_counts = c->selector == SCALECOM_SELECTOR_TOPK;
     return SCALECOM_OK;
 }
 
@@ -788,8 +768,6 @@ int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const i
     lp.n = 1;
     lp.beta = c->beta; lp.omb = 1.0f - c->beta; lp.lr = c->lr; lp.nf = 1.0f;
     lp.bitmap = c->bitmap; lp.bitmap_clear = c->bitmap; lp.tile_prefix = c->tile_prefix;
-    lp.tile_cnt = (!idx && c->select_counts) ? c->tile_cnt : nullptr;   // this handle's own top-k selection left counts
-    lp.group_pre = c->group_pre; lp.gshift = c->gshift;
     lp.out_val = out_gathered; lp.out_idx = c->scratch_idx;
     lp.gathered = nullptr; lp.weights = nullptr; lp.spans = nullptr;
     lp.status = c->ctrl + CT_STATUS;
@@ -799,6 +777,23 @@ int scalecom_compress_scatter(scalecom_ctx* c, const float* g, float* m, const i
                                                          : launch_learner<16, false, LP_ONE_T, 1, true>(c, 1, gp, mp, lp, &peers);
     if (e != cudaSuccess) return SCALECOM_ERR_CUDA;
     ++c->launches;
+    return SCALECOM_OK;
+}
+
+int scalecom_enable_peer_access(scalecom_ctx* c, int32_t peer_device) {
+    if (!c) return SCALECOM_ERR_NULL_PTR;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) { cudaGetLastError(); return SCALECOM_ERR_CUDA; }
+    if (peer_device < 0 || peer_device >= ndev) return SCALECOM_ERR_INVALID_ARG;
+    if (peer_device == c->device) return SCALECOM_OK;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return SCALECOM_ERR_CUDA;
+    int can = 0;
+    if (cudaDeviceCanAccessPeer(&can, c->device, peer_device) != cudaSuccess) { cudaGetLastError(); return SCALECOM_ERR_CUDA; }
+    if (!can) return SCALECOM_ERR_INVALID_ARG;
+    const cudaError_t e = cudaDeviceEnablePeerAccess(peer_device, 0);
+    if (e == cudaErrorPeerAccessAlreadyEnabled) { cudaGetLastError(); return SCALECOM_OK; }
+    if (e != cudaSuccess) { cudaGetLastError(); return SCALECOM_ERR_CUDA; }
     return SCALECOM_OK;
 }
 

@@ -2,42 +2,36 @@
 //
 // Selects the k coordinates of acc = m + g (computed on the fly, never stored)
 // that come first in the order "larger |acc| first, lower index first", and
-// leaves the result as a d-bit bitmap plus two small count arrays from which
-// any consumer derives the rank of a selected coordinate in the ascending index
-// list: the number of selected coordinates of every 1024-coordinate tile, and
-// the exclusive prefix of those counts at the start of every group of tiles.
+// leaves the result in three forms: a d-bit bitmap, the per-tile prefix counts
+// of that bitmap, and the ascending index list.
 //
-// Fast path (one streaming read of g and m, ONE grid barrier):
+// Fast path (one streaming read of g and m):
 //   P0  histogram a strided sample of the keys (top 13 bits)
 //   P1  every block derives from the sample a conservative lower bound on the
 //       k-th key (bin b_lo), aiming at slightly more than k survivors.
-//       P0/P1 (and their barrier) are skipped when earlier launches of the same
-//       handle left a hint: the bin of this leader's k-th key the last time it
-//       led, moved by what the previous step's leader saw change over the same
-//       interval (else the previous step's bin), minus a margin.  A hint that
-//       turns out useless costs one wasted pass; the step then runs P0/P1 as if
-//       there had been none, and later hints keep one more bin of distance
-//   P2  stream g, m once.  16-byte aligned vectors are staged through shared
-//       memory by bulk asynchronous copies (one elected thread issues them, an
-//       mbarrier per stage counts the bytes in, a second one counts the warps
-//       out), so the bytes in flight do not depend on what the warps are doing.
-//       A survivor (key bin >= b_lo) is appended as (key, idx) to a candidate
-//       segment owned by the warp that found it -- no atomics; slots come from a
-//       warp ballot.  Survivor keys also pass through a small per-warp ring from
-//       which, 32 at a time and with all lanes busy, they are added to two
-//       histograms (13-bit bins in a 64-bin window above b_lo, per block in shared
-//       memory; 22-bit prefixes, global)
-//   -- grid barrier --
+//       P0/P1 are skipped when earlier launches of the same handle left a
+//       hint: the bin of this leader's k-th key the last time it led, moved by what the
+//       previous step's leader saw change over the same interval (else the previous
+//       step's bin), minus a margin.  A hint that turns out useless
+//       costs one wasted pass; the step then runs P0/P1 as if there had been none,
+//       and later hints of the handle keep one more bin of distance
+//   P2  stream g, m once.  A survivor (key bin >= b_lo) is appended as (key, idx)
+//       to a candidate segment owned by the warp that found it -- no atomics, no
+//       staging; slots come from a warp ballot.  Survivor keys also pass through a
+//       small per-warp ring in shared memory from which, 32 at a time and with all
+//       lanes busy, they are added to two histograms (13-bit bins in a 64-bin
+//       window above b_lo, per block in shared memory; 22-bit prefixes, global)
 //   P3  the two histograms fix the first 22 bits of the k-th key: candidates
 //       above that prefix are winners, the few hundred sharing it form the
 //       boundary group
-//   P4  every warp marks the winners of its own segment (bitmap bit, tile count,
-//       group total) and appends boundary members to a short global list
-//   P5  blocks count themselves out; the one that finishes last ranks the boundary
-//       list exactly (by key, then lower index), marks its winners, turns the group
-//       totals into prefixes and leaves the scratch arrays clean for the next launch
+//   P4  every warp marks the winners of its own segment in the bitmap and appends
+//       boundary members to a short global list
+//   P5  every block ranks the boundary list exactly (by key, then lower index),
+//       takes the winners that fall in its own span, and prefix-scans its span of
+//       the bitmap: tile prefixes + ascending indices.  The scratch arrays are
+//       cleared here for the next launch
 // A boundary group too large for the short list (heavy ties) is resolved by a
-// radix select over the candidate segments instead (one pass + barrier per digit).
+// radix select over the candidate segments instead (one pass per digit).
 // Exact path (taken when a candidate segment overflowed, too few survived, or
 // the k-th key left the histogram window; also on request): the same radix
 // select with every pass streaming g and m again (up to six passes) and a mark
@@ -51,11 +45,9 @@ constexpr int TK_THREADS = 512;
 constexpr int TK_BLOCKS_PER_SM = 2;
 constexpr int TK_WARPS = TK_THREADS / 32;
 static_assert(TK_WARPS >= 16 && TK_WARPS <= 32, "the block-wide bin search needs 16..32 warps per block");
-constexpr int TK_UNROLL = 4;                                   // quads of g and of m in flight per thread (register path)
-constexpr uint32_t TK_CHUNK = TK_THREADS * 4 * TK_UNROLL;      // coordinates per block iteration of the register path
+constexpr int TK_UNROLL = 4;                        // quads of g and of m in flight per thread
+constexpr uint32_t TK_CHUNK = TK_THREADS * 4 * TK_UNROLL;      // coordinates per block iteration (8192)
 constexpr uint32_t TK_UNIT = TK_THREADS * 4;                   // coordinates one block covers with one quad per thread
-constexpr int TK_STAGES = 6;                                   // shared-memory stages of the filter pass (one unit of g and of m each)
-constexpr uint32_t TK_STAGE_BYTES = 2u * TK_UNIT * 4u;
 
 constexpr int COARSE_SHIFT = 18;                               // key >> 18: 13-bit coarse bin
 constexpr uint32_t NCOARSE = 1u << 13;
@@ -66,23 +58,14 @@ constexpr uint32_t DH_BINS = 2048;                             // digit histogra
 constexpr uint32_t DH_PASSES = 8;
 constexpr uint32_t SAMPLE_GRANULE = 128;                       // coordinates one warp samples at a time
 constexpr uint32_t BCAP = 1024;                                // boundary list entries
-constexpr uint32_t MAX_GROUPS = 4096;                          // groups of tiles (a power-of-two number of tiles each, >= 32)
 
 // ctrl words
 constexpr int CT_CAND = 0, CT_STATUS = 1, CT_PATH = 2, CT_M = 3, CT_BCOUNT = 4, CT_OVERFLOW = 5, CT_HINT = 6, CT_MARGIN = 7;
 constexpr int CT_DRIFT = 21;                                   // (words 8 .. 20 are the phase stamps)
 constexpr int CT_PEER_DONE = 22;                               // finished blocks of a signalling single-learner pass
-constexpr int CT_DONE = 23;                                    // blocks of the selection kernel that are through marking
 constexpr int CT_STAMP = 8, CT_NSTAMPS = 13, CT_WORDS = 32;
 // selection paths reported in ctrl[CT_PATH]
 constexpr uint32_t PATH_FAST = 0, PATH_EXACT = 1, PATH_FAST_HINT = 2;
-
-// Smallest shift s >= 5 with ceil(ntiles / 2^s) <= MAX_GROUPS: a group is 2^s consecutive tiles.
-__host__ __device__ inline uint32_t group_shift_for(uint32_t ntiles) {
-    uint32_t s = 5;
-    while (((ntiles + (1u << s) - 1u) >> s) > MAX_GROUPS) ++s;
-    return s;
-}
 
 struct TopkParams {
     const float* g;            // leader's gradient, fp32[d]
@@ -96,75 +79,37 @@ struct TopkParams {
     uint32_t* all_hints;       // every leader's entry [n_hints] (or nullptr): forgotten when a hint turns out useless
     uint32_t n_hints;
     uint32_t spin_limit;
-    // the histograms, group_tot and the counters in ctrl are all zero on entry and all zero again on exit
+    // the four histograms are all zero on entry and all zero again on exit
     uint32_t* samp_hist;       // [NCOARSE]
     uint32_t* coarse_win;      // [WIN + 1]
     uint32_t* fine_hist;       // [NFINE]
     uint32_t* fine_hist_next;  // [NFINE] the copy the next launch will use, cleared here behind the stream (or nullptr:
                                //         this launch clears its own copy at the end)
     uint32_t* digit_hist;      // [DH_PASSES * DH_BINS]
+    uint32_t* block_tot;       // [gridDim.x] winners per block span
     uint32_t* ctrl;            // [CT_WORDS]
     unsigned long long* barrier;   // arrival counter of the grid barrier
     uint2* cand;               // [seg_cap * warps in the grid] (key, idx), one segment per warp
     uint32_t seg_cap;          // entries per warp segment
     uint2* blist;              // [BCAP] boundary group
-    uint32_t* bitmap;          // [ntiles * 32]                   written
-    uint32_t* tile_cnt;        // [ntiles]  selected coordinates of every tile                      written
-    uint32_t* group_tot;       // [ngroups] scratch
-    uint32_t* group_pre;       // [ngroups + 1] selected coordinates before every group of tiles   written
-    uint32_t ntiles, ngroups, gshift;
+    uint32_t* bitmap;          // [ntiles * 32]
+    uint32_t* tile_prefix;     // [ntiles + 1]
+    uint32_t ntiles;
+    uint32_t tiles_per_block;  // span of the final scan
+    int32_t* out_idx;          // [k], or nullptr when the caller derives the index list itself
     unsigned long long* spans;     // nullptr, or where to accumulate the kernel's time span
 };
 
-struct alignas(128) TopkShared {
-    // stages of the filter pass; outside that pass the first 32 KB serve as histogram / counter scratch
-    float stage[TK_STAGES][2][TK_UNIT];
+struct TopkShared {
+    uint32_t hist[NCOARSE];            // sample histogram / span counters / digit histogram / boundary list
     uint32_t ring[TK_WARPS][64];       // survivor keys waiting for a lane-dense histogram update
     uint32_t cw[WIN + 1];              // this block's share of the coarse window histogram
     uint32_t scan[32];
     uint32_t res[4];
     uint32_t mcount;                   // survivors found by this block
+    uint32_t own_n;                    // boundary winners inside this block's span
     int flag;
-    unsigned long long full_bar[TK_STAGES], empty_bar[TK_STAGES];
 };
-static_assert(sizeof(float) * TK_STAGES * 2 * TK_UNIT >= NCOARSE * 4, "the stages double as the 8192-word scratch");
-
-// ---- bulk asynchronous copies global -> shared with mbarrier completion (this CTA's own shared memory, no multicast) ----
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_addr(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded: a copy that this block issued itself either lands or the kernel gives up (status word, clean exit).
-constexpr uint32_t MBAR_WAIT_LIMIT = 1u << 20;
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
-    for (uint32_t it = 0; it < MBAR_WAIT_LIMIT; ++it)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, unsigned long long* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_addr(smem_dst)),
-                 "l"(gsrc), "r"(bytes), "r"(smem_addr(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Block-wide search from the top of a histogram of nb <= TK_THREADS bins held one bin per thread: thread r holds
 // v = h[nb - 1 - r] (0 for r >= nb).  Finds the bin holding the `need`-th element counted from the top:
@@ -264,10 +209,8 @@ __device__ __forceinline__ bool sel_done(const SelState& st) { return st.group =
 
 template <bool VEC>
 __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kernel(const TopkParams P) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
     TopkShared& s = *reinterpret_cast<TopkShared*>(smem_raw);
-    uint32_t* const hist = reinterpret_cast<uint32_t*>(&s.stage[0][0][0]);   // [NCOARSE] scratch outside the filter pass
-    constexpr bool STAGED = VEC;
 
     const uint32_t tid = threadIdx.x, lane = lane_id(), warp = warp_id();
     const uint32_t nblocks = gridDim.x;
@@ -283,39 +226,27 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
     const uint32_t lt_mask = (1u << lane) - 1u;
 
     // streaming phases: the vector is cut into units of TK_UNIT coordinates dealt round-robin to the
-    // blocks (unit j belongs to block j mod nblocks): block loads differ by at most one unit, and every
-    // block sees every region of the vector (survivors cluster by layer)
+    // blocks (unit j belongs to block j mod nblocks), TK_UNROLL units per block iteration: block loads differ
+    // by at most one unit, and every block sees every region of the vector (survivors cluster by layer)
     const uint32_t nunits = (d + TK_UNIT - 1) / TK_UNIT;
     const uint32_t my_units = nunits > blockIdx.x ? (nunits - blockIdx.x + nblocks - 1) / nblocks : 0u;
     const uint32_t full_units = d / TK_UNIT;                           // units 0 .. full_units-1 need no bounds checks
-    // whole units of this block: those the staged pass fetches with bulk copies
-    const uint32_t my_whole = full_units > blockIdx.x ? (full_units - blockIdx.x + nblocks - 1) / nblocks : 0u;
-    uint32_t stage_seq = 0;                                            // stage uses so far (block-uniform; mbarrier phases follow it)
+    const uint32_t span_coords = P.tiles_per_block * TILE;             // coordinates per block span of the final scan
 
-    // phase time stamps (low word of the nanosecond global timer), for profiling only: 0-7 by block 0, 8-9 by
-    // the block that finishes last
-#define SC_STAMP_IF(cond, i) do { if (cond) { uint32_t ts_; asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(ts_)); \
-                                              P.ctrl[CT_STAMP + (i)] = ts_; } } while (0)
-#define SC_STAMP(i) SC_STAMP_IF(gtid == 0, i)
+    // phase time stamps of block 0 (low word of the nanosecond global timer), for profiling only
+#define SC_STAMP(i) do { if (gtid == 0) { uint32_t ts_; asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(ts_)); \
+                                          P.ctrl[CT_STAMP + (i)] = ts_; } } while (0)
 #define SC_BARRIER() do { if (!grid_barrier(gb, &s.flag)) return; } while (0)
 
     span_begin(P.spans);
     SC_STAMP(0);
     SC_STAMP(1); SC_STAMP(2); SC_STAMP(3);                             // overwritten when the sample phases run
 
-    if (STAGED) {
-        if (tid == 0) {
-#pragma unroll
-            for (int i = 0; i < TK_STAGES; ++i) { mbar_init(&s.full_bar[i], 1u); mbar_init(&s.empty_bar[i], TK_WARPS); }
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
-        __syncthreads();
-    }
-
     // what must be zero before winners are marked; marking starts at least one grid barrier later
     auto clear_outputs = [&] {
         zero_words(P.bitmap, size_t(P.ntiles) * 32, gtid, gsize);
-        zero_words(P.tile_cnt, P.ntiles, gtid, gsize);
+        for (size_t i = gtid; i < nblocks; i += gsize) P.block_tot[i] = 0;
+        if (gtid == 0) P.ctrl[CT_BCOUNT] = 0;
         if (P.fine_hist_next) zero_words(P.fine_hist_next, NFINE, gtid, gsize);
     };
 
@@ -349,7 +280,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                 for (size_t i = gtid; i <= WIN; i += gsize) P.coarse_win[i] = 0;
                 if (gtid == 0) { P.ctrl[CT_CAND] = 0; P.ctrl[CT_OVERFLOW] = 0; }
             }
-            for (uint32_t i = tid; i < NCOARSE; i += TK_THREADS) hist[i] = 0;
+            for (uint32_t i = tid; i < NCOARSE; i += TK_THREADS) s.hist[i] = 0;
             __syncthreads();
             const uint32_t span = SAMPLE_GRANULE * P.samp_stride;      // coordinates between sampled granules
             const uint32_t ngran = (d + span - 1) / span;
@@ -360,11 +291,11 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                 load_quad_stream<VEC>(P.m, p, d, mv);
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    if (p + c < d) atomicAdd(&hist[mag_key(__fadd_rn(mv[c], gv[c])) >> COARSE_SHIFT], 1u);
+                    if (p + c < d) atomicAdd(&s.hist[mag_key(__fadd_rn(mv[c], gv[c])) >> COARSE_SHIFT], 1u);
             }
             __syncthreads();
             for (uint32_t i = tid; i < NCOARSE; i += TK_THREADS) {
-                const uint32_t h = hist[i];
+                const uint32_t h = s.hist[i];
                 if (h) atomicAdd(&P.samp_hist[i], h);
             }
             SC_STAMP(1);
@@ -379,27 +310,10 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
         b_lo = min(b_lo, 0x7F800000u >> COARSE_SHIFT);                 // at most the bin of +inf: the bound stays a number
 
         // ---------------- P2: filter pass ----------------------------------------------------------
+        clear_outputs();                                               // hidden behind the stream
         for (uint32_t i = tid; i <= WIN; i += TK_THREADS) s.cw[i] = 0;
         if (tid == 0) s.mcount = 0;
-        __syncthreads();                                               // (also: nobody still uses the scratch the stages overlay)
-        // request the first stages before anything else is done
-        uint32_t n_issued = 0;                                         // (thread 0) units requested in this pass
-        auto issue = [&](uint32_t it) {                                // thread 0 only: fetch this block's it-th unit
-            const uint32_t q = stage_seq + it, sg = q % TK_STAGES, round = q / TK_STAGES;
-            bool free_ = true;
-            if (round > 0) free_ = mbar_wait(&s.empty_bar[sg], (round - 1u) & 1u);   // every warp is through with the previous use
-            if (!free_) { atomicCAS(status, DEV_OK, DEV_TIMEOUT); return; }
-            const size_t p = size_t(it * nblocks + blockIdx.x) * TK_UNIT;
-            mbar_expect_tx(&s.full_bar[sg], TK_STAGE_BYTES);
-            bulk_load(&s.stage[sg][0][0], P.g + p, TK_UNIT * 4u, &s.full_bar[sg]);
-            bulk_load(&s.stage[sg][1][0], P.m + p, TK_UNIT * 4u, &s.full_bar[sg]);
-            ++n_issued;
-        };
-        if (STAGED && tid == 0) {
-            fence_async_smem();                                        // generic-proxy writes to the scratch come first
-            for (uint32_t it = 0; it < uint32_t(TK_STAGES - 1) && it < my_whole; ++it) issue(it);
-        }
-        clear_outputs();                                               // hidden behind the stream
+        __syncthreads();
         seg_cnt = 0;
         uint32_t done = 0;                                             // survivors of this warp already histogrammed
         const uint32_t thr_key = b_lo << COARSE_SHIFT;
@@ -437,43 +351,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                 bal = __ballot_sync(FULL, nib != 0);
             }
         };
-        auto filter_quad = [&](const float (&gq)[4], const float (&mq)[4], uint32_t p, bool checked) {
-            float acc[4];
-            uint32_t nib = 0;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                acc[c] = __fadd_rn(mq[c], gq[c]);
-                if ((!checked || p + c < d) && !(fabsf(acc[c]) < thr_f)) nib |= 1u << c;
-            }
-            append(nib, acc, p);
-        };
-        uint32_t it_first = 0;                                         // first unit the register path has to take
-        if (STAGED) {
-            bool alive = true;
-            uint32_t it = 0;
-            for (; it < my_whole; ++it) {
-                if (tid == 0 && it + uint32_t(TK_STAGES - 1) < my_whole) issue(it + uint32_t(TK_STAGES - 1));
-                const uint32_t q = stage_seq + it, sg = q % TK_STAGES;
-                alive = __all_sync(FULL, mbar_wait(&s.full_bar[sg], (q / TK_STAGES) & 1u));
-                if (!alive) break;                                     // (the same for every warp: they wait for the same copy)
-                const float4 a = *reinterpret_cast<const float4*>(&s.stage[sg][0][tid * 4]);
-                const float4 b = *reinterpret_cast<const float4*>(&s.stage[sg][1][tid * 4]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&s.empty_bar[sg]);          // this warp holds its part of the stage in registers
-                const float gq[4] = {a.x, a.y, a.z, a.w}, mq[4] = {b.x, b.y, b.z, b.w};
-                filter_quad(gq, mq, (it * nblocks + blockIdx.x) * TK_UNIT + tid * 4, false);
-            }
-            if (!alive && tid == 0) {
-                // give up: the grid barrier below sees the status word and everybody leaves -- but not before this
-                // block's own copies have landed (bounded again), since they write into its shared memory
-                atomicCAS(status, DEV_OK, DEV_TIMEOUT);
-                for (uint32_t o = it; o < n_issued; ++o)
-                    mbar_wait(&s.full_bar[(stage_seq + o) % TK_STAGES], ((stage_seq + o) / TK_STAGES) & 1u);
-            }
-            stage_seq += my_whole;
-            it_first = my_whole;
-        }
-        for (uint32_t it0 = it_first; it0 < my_units; it0 += TK_UNROLL) {
+        for (uint32_t it0 = 0; it0 < my_units; it0 += TK_UNROLL) {
             float gv[TK_UNROLL][4], mv[TK_UNROLL][4];
             const bool whole = VEC && it0 + TK_UNROLL <= my_units &&
                                (it0 + TK_UNROLL - 1) * nblocks + blockIdx.x < full_units;
@@ -488,7 +366,17 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                     mv[u][0] = b.x; mv[u][1] = b.y; mv[u][2] = b.z; mv[u][3] = b.w;
                 }
 #pragma unroll
-                for (int u = 0; u < TK_UNROLL; ++u) filter_quad(gv[u], mv[u], pbase + u * (nblocks * TK_UNIT), false);
+                for (int u = 0; u < TK_UNROLL; ++u) {
+                    const uint32_t p = pbase + u * (nblocks * TK_UNIT);
+                    float acc[4];
+                    uint32_t nib = 0;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        acc[c] = __fadd_rn(mv[u][c], gv[u][c]);
+                        if (!(fabsf(acc[c]) < thr_f)) nib |= 1u << c;
+                    }
+                    append(nib, acc, p);
+                }
             } else {
 #pragma unroll
                 for (int u = 0; u < TK_UNROLL; ++u) {
@@ -496,8 +384,17 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                     if (p < d) { load_quad_stream<VEC>(P.g, p, d, gv[u]); load_quad_stream<VEC>(P.m, p, d, mv[u]); }
                 }
 #pragma unroll
-                for (int u = 0; u < TK_UNROLL; ++u)
-                    filter_quad(gv[u], mv[u], unit_coord(it0 + u, my_units, nblocks, d) + tid * 4, true);
+                for (int u = 0; u < TK_UNROLL; ++u) {
+                    const uint32_t p = unit_coord(it0 + u, my_units, nblocks, d) + tid * 4;
+                    float acc[4];
+                    uint32_t nib = 0;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        acc[c] = __fadd_rn(mv[u][c], gv[u][c]);
+                        if ((p + c < d) && !(fabsf(acc[c]) < thr_f)) nib |= 1u << c;
+                    }
+                    append(nib, acc, p);
+                }
             }
         }
         if (seg_cnt > done) drain(seg_cnt - done);
@@ -557,7 +454,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
         P.ctrl[CT_M] = M;
     }
 
-    // a small boundary group is ranked by the last block; anything else goes digit by digit
+    // a small boundary group is ranked in P5; anything else goes digit by digit
     const bool boundary = fast && !sel_done(st) && st.nbits == 22 && st.group <= BCAP;
     uint32_t pass = 0;
     while (!boundary && !sel_done(st)) {
@@ -576,7 +473,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                 if ((c >> shift_match) == st.prefix) atomicAdd(&gh[uint32_t(c >> shift_digit) & dmask], 1u);
             }
         } else {
-            for (uint32_t i = tid; i < DH_BINS; i += TK_THREADS) hist[i] = 0;
+            for (uint32_t i = tid; i < DH_BINS; i += TK_THREADS) s.hist[i] = 0;
             __syncthreads();
             for (uint32_t it0 = 0; it0 < my_units; it0 += TK_UNROLL) {
                 float gv[TK_UNROLL][4], mv[TK_UNROLL][4];
@@ -596,14 +493,14 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                         if (pr) {
                             const uint32_t dg = uint32_t(cc >> shift_digit) & dmask;
                             const uint32_t peers = __match_any_sync(act, dg);
-                            if (lane == uint32_t(__ffs(peers) - 1)) atomicAdd(&hist[dg], uint32_t(__popc(peers)));
+                            if (lane == uint32_t(__ffs(peers) - 1)) atomicAdd(&s.hist[dg], uint32_t(__popc(peers)));
                         }
                     }
                 }
             }
             __syncthreads();
             for (uint32_t i = tid; i < DH_BINS; i += TK_THREADS) {
-                const uint32_t h = hist[i];
+                const uint32_t h = s.hist[i];
                 if (h) atomicAdd(&gh[i], h);
             }
         }
@@ -626,46 +523,25 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
     // winners are the composites >= T; with a boundary group, T covers it and the group is ranked separately
     const uint64_t T = st.nbits >= 62 ? st.prefix : (st.prefix << (62 - st.nbits));
     const uint64_t T_above = boundary ? ((st.prefix + 1) << (62 - st.nbits)) : T;   // strictly above the group
-    const uint32_t gshift = P.gshift;
-    // winners per group of tiles are counted in shared memory first
-    for (uint32_t i = tid; i < P.ngroups; i += TK_THREADS) hist[i] = 0;
-    __syncthreads();
-    SC_STAMP(10);
     if (fast) {
-        // A warp's survivors of one visit lie within 128 consecutive coordinates, and where one coordinate passes the
-        // pre-filter its neighbours tend to as well: winners of the same bitmap word / tile among the 32 entries in
-        // hand are combined first, so that a dense tile costs its address a few atomics, not hundreds
-        constexpr int MB = 4;                                          // entries per lane requested at a time
-        for (uint32_t i0 = 0; i0 < seg_cnt; i0 += 32 * MB) {
-            uint2 ent[MB];
-#pragma unroll
-            for (int j = 0; j < MB; ++j) {
-                const uint32_t i = i0 + j * 32 + lane;
-                ent[j] = i < seg_cnt ? __ldcg(&seg[i]) : make_uint2(0u, 0u);
+        // winners per scan span are counted in shared memory first (nblocks <= NCOARSE spans)
+        for (uint32_t i = tid; i < nblocks; i += TK_THREADS) s.hist[i] = 0;
+        __syncthreads();
+        for (uint32_t i = lane; i < seg_cnt; i += 32) {
+            const uint2 e = __ldcg(&seg[i]);
+            const uint64_t c = composite(e.x, e.y);
+            if (c >= T_above) {
+                atomicOr(&P.bitmap[e.y >> 5], 1u << (e.y & 31u));
+                atomicAdd(&s.hist[e.y / span_coords], 1u);
+            } else if (c >= T) {                                       // only with a boundary group
+                const uint32_t slot = atomicAdd(&P.ctrl[CT_BCOUNT], 1u);
+                if (slot < BCAP) P.blist[slot] = e;
             }
-#pragma unroll
-            for (int j = 0; j < MB; ++j) {
-                if (i0 + j * 32 >= seg_cnt) break;                     // warp-uniform
-                const uint32_t i = i0 + j * 32 + lane;
-                const uint2 e = ent[j];
-                const uint64_t c = composite(e.x, e.y);
-                const bool winner = i < seg_cnt && c >= T_above;
-                const uint32_t wmask = __ballot_sync(FULL, winner);
-                if (winner) {
-                    const uint32_t word = e.y >> 5, tile = e.y / TILE;
-                    const uint32_t same_word = __match_any_sync(wmask, word);
-                    const uint32_t bits = __reduce_or_sync(same_word, 1u << (e.y & 31u));
-                    if (lane == uint32_t(__ffs(same_word) - 1)) atomicOr(&P.bitmap[word], bits);
-                    const uint32_t same_tile = __match_any_sync(wmask, tile);
-                    if (lane == uint32_t(__ffs(same_tile) - 1)) {
-                        atomicAdd(&P.tile_cnt[tile], uint32_t(__popc(same_tile)));
-                        atomicAdd(&hist[tile >> gshift], uint32_t(__popc(same_tile)));
-                    }
-                } else if (i < seg_cnt && c >= T) {                    // only with a boundary group
-                    const uint32_t slot = atomicAdd(&P.ctrl[CT_BCOUNT], 1u);
-                    if (slot < BCAP) P.blist[slot] = e;
-                }
-            }
+        }
+        __syncthreads();
+        for (uint32_t i = tid; i < nblocks; i += TK_THREADS) {
+            const uint32_t h = s.hist[i];
+            if (h) atomicAdd(&P.block_tot[i], h);
         }
     } else {
         // every 128-coordinate group is owned by one warp: whole bitmap words, plain stores
@@ -693,49 +569,43 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                 const uint32_t p0 = p - lane * 4;                      // first coordinate of the warp's 128
                 if (p0 < d) {
                     if ((lane & 7u) == 0) P.bitmap[(p0 >> 5) + (lane >> 3)] = word;
-                    if (lane == 0 && wsum) {
-                        atomicAdd(&P.tile_cnt[p0 / TILE], wsum);
-                        atomicAdd(&hist[(p0 / TILE) >> gshift], wsum);
-                    }
+                    if (lane == 0 && wsum) atomicAdd(&P.block_tot[p0 / span_coords], wsum);
                 }
             }
         }
     }
-    SC_STAMP(11);
-    __syncthreads();
-    SC_STAMP(12);
-    for (uint32_t i = tid; i < P.ngroups; i += TK_THREADS) {
-        const uint32_t h = hist[i];
-        if (h) atomicAdd(&P.group_tot[i], h);
-    }
     SC_STAMP(7);
+    SC_BARRIER();
+    SC_STAMP(8);
 
-    // ---------------- P5: the block that finishes last completes the result -------------------------------
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        s.flag = atomicAdd(&P.ctrl[CT_DONE], 1u) == nblocks - 1u;
-        __threadfence();
-    }
-    __syncthreads();
-    if (s.flag) {
-        SC_STAMP_IF(tid == 0, 8);
-        // shared-memory scratch: group totals, histogram of the boundary members' last 9 key bits, members on the k-th key
-        uint32_t* gs = hist;                                           // [MAX_GROUPS]
-        uint32_t* kh = gs + MAX_GROUPS;                                // [512]
-        uint32_t* ties = kh + 512;                                     // [BCAP]
-        const uint32_t ngroups = P.ngroups;
-        for (uint32_t i = tid; i < MAX_GROUPS; i += TK_THREADS) {
-            const bool live = i < ngroups;
-            gs[i] = live ? __ldcg(&P.group_tot[i]) : 0u;
-            if (live) P.group_tot[i] = 0u;                             // zero again for the next launch
-        }
+    // ---------------- P5: boundary group, scan of the bitmap, clean-up ----------------------------------
+    {
+        // each warp owns a contiguous run of the span's tiles; all loads of this phase are issued up front
+        const uint32_t t0 = blockIdx.x * P.tiles_per_block;
+        const uint32_t t1 = min(P.ntiles, t0 + P.tiles_per_block);
+        const uint32_t nt = t1 > t0 ? t1 - t0 : 0u;
+        const uint32_t per_warp = (nt + TK_WARPS - 1) / TK_WARPS;
+        const uint32_t w0 = min(t1, t0 + warp * per_warp), w1 = min(t1, w0 + per_warp);
+        constexpr int RW = 8;                                          // tiles per warp kept in registers
+        uint32_t wreg[RW];
+#pragma unroll
+        for (int j = 0; j < RW; ++j) wreg[j] = (w0 + j < w1) ? __ldcg(&P.bitmap[size_t(w0 + j) * 32 + lane]) : 0u;
+        uint32_t part = 0;                                             // winners before this block's span
+        for (uint32_t b = tid; b < blockIdx.x; b += TK_THREADS) part += __ldcg(&P.block_tot[b]);
+
+        // shared-memory scratch carved from the (idle) histogram array
+        uint32_t* own = s.hist;                                        // [BCAP] boundary winners inside this block's span
+        uint32_t* kh = own + BCAP;                                     // [512]  histogram of the members' last 9 key bits
+        uint32_t* ties = kh + 512;                                     // [BCAP] members sharing the k-th key
+        if (tid == 0) { s.own_n = 0; s.res[3] = 0; }
         if (boundary) {
-            // The members share 22 key bits; a 512-bin histogram of the remaining 9 finds the k-th key, members
-            // above it win, members on it are ranked by index among themselves (all composites are distinct, so
-            // the answer is unique).
+            // Every block ranks the boundary group itself.  The members share 22 key bits; a 512-bin
+            // histogram of the remaining 9 finds the k-th key, members above it win, members on it are
+            // ranked by index among themselves.  Winners inside this block's span are kept in `own`
+            // (and set in the global bitmap for the learner pass), winners before it are counted.
             const uint32_t cnt = st.group;                             // <= BCAP
-            if (tid == 0) { s.res[3] = 0; if (__ldcg(&P.ctrl[CT_BCOUNT]) != cnt) atomicCAS(status, DEV_OK, DEV_INTERNAL); }
+            if (tid == 0 && __ldcg(&P.ctrl[CT_BCOUNT]) != cnt)         // cannot happen: the histograms counted `group`
+                atomicCAS(status, DEV_OK, DEV_INTERNAL);
             for (uint32_t i = tid; i < 512; i += TK_THREADS) kh[i] = 0;
             uint2 mine[BCAP / TK_THREADS];
 #pragma unroll
@@ -764,11 +634,14 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
             }
             __syncthreads();
             const uint32_t kstar = s.res[0], need_ties = st.need - s.res[1];
+            const uint32_t c0 = blockIdx.x * span_coords;
             auto win = [&](uint32_t idx) {
-                const uint32_t tile = idx / TILE;
-                atomicOr(&P.bitmap[idx >> 5], 1u << (idx & 31u));
-                atomicAdd(&P.tile_cnt[tile], 1u);
-                atomicAdd(&gs[tile >> gshift], 1u);
+                if (idx < c0) {
+                    ++part;
+                } else if (idx - c0 < span_coords) {
+                    atomicOr(&P.bitmap[idx >> 5], 1u << (idx & 31u));   // for the learner pass; not read back here
+                    own[atomicAdd(&s.own_n, 1u)] = idx;
+                }
             };
 #pragma unroll
             for (int r = 0; r < int(BCAP / TK_THREADS); ++r)
@@ -787,47 +660,85 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
             }
         }
         __syncthreads();
-        // exclusive prefix of the group totals: consecutive groups per thread, then across the block
-        constexpr uint32_t PER = MAX_GROUPS / TK_THREADS;
-        uint32_t loc[PER], tot = 0;
+        SC_STAMP(10);
+        const uint32_t own_n = s.own_n;
+        // bitmap word (tile, lane) with this block's boundary winners merged in
+        auto merge_own = [&](uint32_t tile, uint32_t word) {
+            for (uint32_t o = 0; o < own_n; ++o) {
+                const uint32_t idx = own[o];
+                if ((idx >> 5) == tile * 32 + lane) word |= 1u << (idx & 31u);
+            }
+            return word;
+        };
+        uint32_t ttot[RW];                                             // winners per cached tile
+        uint32_t wtot = 0;
 #pragma unroll
-        for (uint32_t j = 0; j < PER; ++j) { loc[j] = gs[tid * PER + j]; tot += loc[j]; }
-        const uint32_t incl = warp_incl_scan(tot);
-        if (lane == 31) s.scan[warp] = incl;
-        __syncthreads();
-        uint32_t run = incl - tot;
-#pragma unroll
-        for (int w = 0; w < TK_WARPS; ++w)
-            if (w < (int)warp) run += s.scan[w];
-#pragma unroll
-        for (uint32_t j = 0; j < PER; ++j) {
-            const uint32_t i = tid * PER + j;
-            if (i <= ngroups) P.group_pre[i] = run;                    // entry ngroups: the grand total
-            run += loc[j];
+        for (int j = 0; j < RW; ++j) {
+            if (own_n && w0 + j < w1) wreg[j] = merge_own(w0 + j, wreg[j]);
+            ttot[j] = __reduce_add_sync(FULL, uint32_t(__popc(wreg[j])));
+            wtot += ttot[j];
         }
-        if (tid == TK_THREADS - 1) {
-            if (ngroups == MAX_GROUPS) P.group_pre[MAX_GROUPS] = run;
-            if (run != k) atomicCAS(status, DEV_OK, DEV_INTERNAL);     // the winners must number exactly k
+        for (uint32_t tile = w0 + RW; tile < w1; ++tile)
+            wtot += __reduce_add_sync(FULL, uint32_t(__popc(merge_own(tile, __ldcg(&P.bitmap[size_t(tile) * 32 + lane])))));
+        part = __reduce_add_sync(FULL, part);
+        if (lane == 0) { s.scan[warp] = wtot; s.cw[warp] = part; }
+        __syncthreads();
+        SC_STAMP(11);
+        uint32_t running = 0;                                          // winners before this warp's run
+#pragma unroll
+        for (int w = 0; w < TK_WARPS; ++w) {
+            running += s.cw[w];
+            if (w < (int)warp) running += s.scan[w];
+        }
+        // per tile: its prefix count, and (when asked for) its indices in ascending order
+        auto emit = [&](uint32_t tile, uint32_t word, uint32_t total) {
+            if (lane == 0) P.tile_prefix[tile] = running;
+            if (P.out_idx) {
+                const uint32_t cnt = __popc(word);
+                uint32_t off = running + warp_incl_scan(cnt) - cnt;
+                const uint32_t cbase = tile * TILE + lane * 32;
+                while (word) {
+                    const uint32_t b = __ffs(word) - 1;
+                    word &= word - 1;
+                    if (off < k) P.out_idx[off] = int32_t(cbase + b);
+                    ++off;
+                }
+            }
+            running += total;
+        };
+#pragma unroll
+        for (int j = 0; j < RW; ++j)
+            if (w0 + j < w1) emit(w0 + j, wreg[j], ttot[j]);
+        for (uint32_t tile = w0 + RW; tile < w1; ++tile) {
+            const uint32_t word = merge_own(tile, __ldcg(&P.bitmap[size_t(tile) * 32 + lane]));
+            emit(tile, word, __reduce_add_sync(FULL, uint32_t(__popc(word))));
+        }
+        if (blockIdx.x == nblocks - 1 && tid == TK_THREADS - 1) {
+            // the last warp of the last block ends on the grand total: the winners must number exactly k
+            P.tile_prefix[P.ntiles] = running;
+            if (running != k) atomicCAS(status, DEV_OK, DEV_INTERNAL);
         }
 
+        SC_STAMP(12);
         // leave the histograms and counters zero for the next launch, and the hint for its bound
-        if (!P.fine_hist_next) zero_words(P.fine_hist, NFINE, tid, TK_THREADS);
-        for (uint32_t i = tid; i <= WIN; i += TK_THREADS) P.coarse_win[i] = 0;
-        if (pass) zero_words(P.digit_hist, size_t(pass) * DH_BINS, tid, TK_THREADS);
-        if (tid == 0) {
-            P.ctrl[CT_CAND] = 0; P.ctrl[CT_OVERFLOW] = 0; P.ctrl[CT_BCOUNT] = 0; P.ctrl[CT_DONE] = 0;
+        if (!P.fine_hist_next) zero_words(P.fine_hist, NFINE, gtid, gsize);
+        for (size_t i = gtid; i <= WIN; i += gsize) P.coarse_win[i] = 0;
+        if (pass) zero_words(P.digit_hist, size_t(pass) * DH_BINS, gtid, gsize);
+        if (gtid == 0) {
+            P.ctrl[CT_CAND] = 0; P.ctrl[CT_OVERFLOW] = 0;
         }
-        if (tid == 0 && P.use_hint) {
+        if (gtid == 0 && P.use_hint) {
             // the 13-bit bin (about 3 % in magnitude) of the k-th key just found, for this leader and for the next
             // step.  Later bounds keep one bin of distance; two after a hint that left too few survivors, one again
             // after one that left too many or came close to it (error feedback piles coordinates up just below
             // the threshold: late in a run one bin holds about k of them)
             if (hint && !used_hint) P.ctrl[CT_MARGIN] = hint_overflowed ? 0u : 1u;
             else if (used_hint && M > 3u * k) P.ctrl[CT_MARGIN] = 0u;
-            // a useless hint means the scale moved under every learner: what the other leaders remember (and the
-            // change this one is about to record against its own stale value) would mislead the next steps, which
-            // start from this step's bin instead until each leader has led again
-            const bool forget = hint && !used_hint && P.all_hints;
+            // a useless hint that came from this leader's own earlier value means the scale moved under the learners:
+            // what the other leaders remember (and the change this one is about to record against its stale value)
+            // would mislead the next steps, which start from this step's bin instead until each leader has led
+            // again.  (A useless hint borrowed from the previous step's leader only says that learners differ.)
+            const bool forget = hint && !used_hint && own_prev && P.all_hints;
             if (forget)
                 for (uint32_t i = 0; i < P.n_hints; ++i) P.all_hints[i] = 0u;
             const uint32_t cbk = st.nbits >= 13 ? uint32_t(st.prefix >> (st.nbits - 13)) : 0u;
@@ -836,36 +747,11 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
             P.ctrl[CT_HINT] = cbk ? cbk + 1u : 0u;
             if (P.leader_hint) *P.leader_hint = cbk ? cbk + 1u : 0u;
         }
-        SC_STAMP_IF(tid == 0, 9);
     }
+    SC_STAMP(9);
     span_end(P.spans);
 #undef SC_BARRIER
 #undef SC_STAMP
-#undef SC_STAMP_IF
-}
-
-// The ascending index list from the selection's bitmap and counts: one warp per tile.
-static __global__ void __launch_bounds__(256) emit_indices_kernel(const uint32_t* __restrict__ bitmap,
-                                                           const uint32_t* __restrict__ tile_cnt,
-                                                           const uint32_t* __restrict__ group_pre, uint32_t gshift,
-                                                           uint32_t ntiles, uint32_t k, int32_t* __restrict__ out_idx,
-                                                           const uint32_t* __restrict__ status) {
-    if (ld_relaxed_u32(status) != DEV_OK) return;                      // no valid selection after a device error
-    const uint32_t lane = lane_id();
-    const uint32_t wpg = (gridDim.x * blockDim.x) >> 5;
-    for (uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; tile < ntiles; tile += wpg) {
-        uint32_t word = __ldg(bitmap + size_t(tile) * 32 + lane);
-        if (__ballot_sync(FULL, word != 0u) == 0u) continue;
-        const uint32_t cnt = __popc(word);
-        uint32_t off = selected_before_tile(tile_cnt, group_pre, gshift, tile) + warp_incl_scan(cnt) - cnt;
-        const uint32_t cbase = tile * TILE + lane * 32;
-        while (word) {
-            const uint32_t b = __ffs(word) - 1;
-            word &= word - 1;
-            if (off < k) out_idx[off] = int32_t(cbase + b);
-            ++off;
-        }
-    }
 }
 
 }  // namespace sc

@@ -30,14 +30,13 @@ constexpr size_t OFF_SAMP = 0;
 constexpr size_t OFF_CW = OFF_SAMP + al(NCOARSE * 4);
 constexpr size_t OFF_CTRL = OFF_CW + al((WIN + 1) * 4);
 constexpr size_t OFF_BAR = OFF_CTRL + al(CT_WORDS * 4);
-constexpr size_t OFF_GT = OFF_BAR + al(256);
-constexpr size_t OFF_FINE = OFF_GT + al(size_t(MAX_GROUPS) * 4);
+constexpr size_t OFF_BT = OFF_BAR + al(256);
+constexpr size_t OFF_FINE = OFF_BT + al(MAX_BLOCKS * 4);
 constexpr size_t OFF_DH = OFF_FINE + al(NFINE * 4);
 constexpr size_t OFF_CLEAR_END = OFF_DH + al(size_t(DH_PASSES) * DH_BINS * 4);
 constexpr size_t OFF_BM = OFF_CLEAR_END;
-constexpr size_t OFF_TC = OFF_BM + al(size_t(MAX_TILES) * 32 * 4);
-constexpr size_t OFF_GP = OFF_TC + al(size_t(MAX_TILES) * 4);
-constexpr size_t OFF_BL = OFF_GP + al((size_t(MAX_GROUPS) + 1) * 4);
+constexpr size_t OFF_TP = OFF_BM + al(size_t(MAX_TILES) * 32 * 4);
+constexpr size_t OFF_BL = OFF_TP + al((size_t(MAX_TILES) + 1) * 4);
 constexpr size_t OFF_CAND = OFF_BL + al(size_t(BCAP) * 8);
 constexpr size_t CAND_ENTRIES = size_t(MAX_D) + 32u * MAX_BLOCKS * TK_WARPS;   // every warp's share of the vector + slack
 constexpr size_t SCRATCH_BYTES = OFF_CAND + al(CAND_ENTRIES * 8);
@@ -136,18 +135,15 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
     P.coarse_win = reinterpret_cast<uint32_t*>(base + OFF_CW);
     P.ctrl = reinterpret_cast<uint32_t*>(base + OFF_CTRL);
     P.barrier = reinterpret_cast<unsigned long long*>(base + OFF_BAR);
-    P.group_tot = reinterpret_cast<uint32_t*>(base + OFF_GT);
+    P.block_tot = reinterpret_cast<uint32_t*>(base + OFF_BT);
     P.fine_hist = reinterpret_cast<uint32_t*>(base + OFF_FINE);
     P.fine_hist_next = nullptr;   // one copy: the memset before every launch clears it
     P.digit_hist = reinterpret_cast<uint32_t*>(base + OFF_DH);
     P.bitmap = reinterpret_cast<uint32_t*>(base + OFF_BM);
-    P.tile_cnt = reinterpret_cast<uint32_t*>(base + OFF_TC);
-    P.group_pre = reinterpret_cast<uint32_t*>(base + OFF_GP);
+    P.tile_prefix = reinterpret_cast<uint32_t*>(base + OFF_TP);
     P.cand = reinterpret_cast<uint2*>(base + OFF_CAND);
     P.blist = reinterpret_cast<uint2*>(base + OFF_BL);
     P.ntiles = uint32_t((d + TILE - 1) / TILE);
-    P.gshift = group_shift_for(P.ntiles);
-    P.ngroups = (P.ntiles + (1u << P.gshift) - 1u) >> P.gshift;
     const uint32_t chunks = uint32_t((d + TK_CHUNK - 1) / TK_CHUNK);
     uint32_t blocks = uint32_t(su.max_blocks);
     if (blocks > chunks) blocks = chunks;
@@ -161,6 +157,8 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
         if (cap * warps > int64_t(CAND_ENTRIES)) cap = int64_t(CAND_ENTRIES) / warps;
         P.seg_cap = uint32_t(cap);
     }
+    P.tiles_per_block = (P.ntiles + blocks - 1) / blocks;
+    P.out_idx = out_idx;
     P.spans = nullptr;
 
     // Every call shares the array and finds the previous call's contents in it: the
@@ -174,13 +172,6 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
     if (cudaLaunchCooperativeKernel(fn, dim3(blocks), dim3(TK_THREADS), args, sizeof(TopkShared), stream) != cudaSuccess) {
         cudaGetLastError();
         return SCALECOM_ERR_CUDA;
-    }
-    // the ascending list from the bitmap and the counts the selection left in the array
-    {
-        const uint32_t want = (P.ntiles + 7u) / 8u;
-        emit_indices_kernel<<<want < 1024u ? want : 1024u, 256, 0, stream>>>(P.bitmap, P.tile_cnt, P.group_pre, P.gshift,
-                                                                             P.ntiles, P.k, out_idx, P.ctrl + CT_STATUS);
-        if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
     }
     if (dev_status &&
         cudaMemcpyAsync(dev_status, P.ctrl + CT_STATUS, 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {

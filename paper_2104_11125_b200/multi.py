@@ -31,11 +31,19 @@ rank's flag words (bounded; TIMEOUT in the handle's status when a sender never a
 rows.  The index broadcast is then the only collective of the step.  Here a kernel does wait for other ranks'
 kernels, so the ranks must be on different GPUs.
 
+Both peer forms store through pointers into other GPUs' memory, which is only legal once the storing
+device has peer access to the owning device.  Before anything is mapped, every rank therefore checks that
+each peer on another device of the same host is reachable (torch.cuda.can_device_access_peer) and enables
+the access explicitly with scalecom_enable_peer_access; the ranks agree on the outcome, and if any pair lacks
+access (or a peer sits on another host) all of them fall back to exchange="collective" with a warning.
+
 This module only orders calls; all arithmetic is in the library's kernels.
 """
 from __future__ import annotations
 
-from typing import Optional, Sequence, Tuple
+import socket
+import warnings
+from typing import Callable, Optional, Sequence, Tuple
 
 import torch
 import torch.distributed as dist
@@ -49,7 +57,8 @@ class LearnerRank:
 
     def __init__(self, d: int, k: int, beta: float, lr: float, group: Optional[dist.ProcessGroup] = None,
                  selector: int = binding.SELECTOR_TOPK, layers: Optional[Tuple[Sequence[int], Sequence[int]]] = None,
-                 engine=None, device: Optional[torch.device] = None, exchange: str = "collective"):
+                 engine=None, device: Optional[torch.device] = None, exchange: str = "collective",
+                 can_access_peer: Optional[Callable[[int, int], bool]] = None):
         if not dist.is_initialized():
             raise RuntimeError("torch.distributed must be initialised before a LearnerRank is made")
         self.group = group
@@ -72,10 +81,37 @@ class LearnerRank:
         if exchange not in ("collective", "peer", "peer-flags"):
             raise ValueError("exchange must be 'collective', 'peer' or 'peer-flags'")
         self.exchange = exchange
+        self._can_access_peer = can_access_peer if can_access_peer is not None else torch.cuda.can_device_access_peer
         if exchange != "collective":
-            if not isinstance(self.engine, binding.Context):
-                raise ValueError("exchange='peer' needs the CUDA engine")
-            self._map_peer_rows(dev)
+            peer_devices = self._reachable_peer_devices(dev)
+            if peer_devices is None:
+                warnings.warn("scalecom: exchange=%r needs peer access between all ranks' devices on one host; "
+                              "at least one pair lacks it, every rank falls back to exchange='collective'" % exchange)
+                self.exchange = "collective"
+            else:
+                if not isinstance(self.engine, binding.Context):
+                    raise ValueError("exchange='peer' needs the CUDA engine")
+                for other in peer_devices:                  # the device whose kernels store gets the access
+                    self.engine.enable_peer_access(other)
+                self._map_peer_rows(dev)
+
+    def _reachable_peer_devices(self, dev: torch.device):
+        """The other devices this rank's kernels would store to (device indices, same host), or None when any rank
+        of the group reports a peer it cannot reach.  Every rank returns None together."""
+        mine = (socket.gethostname(), dev.type, dev.index if dev.index is not None else -1 - self.rank)
+        keys = [None] * self.world
+        dist.all_gather_object(keys, mine, group=self.group)
+        others, ok = [], True
+        for r, (host, kind, index) in enumerate(keys):
+            if r == self.rank or (host, kind, index) == mine:
+                continue                                    # this rank, or a rank sharing this device
+            if host != mine[0] or kind != "cuda" or mine[1] != "cuda" or not self._can_access_peer(mine[2], index):
+                ok = False
+            elif index not in others:
+                others.append(index)
+        verdicts = [None] * self.world
+        dist.all_gather_object(verdicts, ok, group=self.group)
+        return others if all(verdicts) else None
 
     def _map_peer_rows(self, dev: torch.device) -> None:
         """Two gathered-rows buffers [2][world][k] per rank and their flag words [2][world], each mapped into

@@ -1,6 +1,6 @@
 """One rank of a learner-per-process job, run as a child process by test_exchange.py.
 
-usage: exchange_worker.py <cpu|gpu|gpu-peer|gpu-flags> <topk|chunk|layer_topk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
+usage: exchange_worker.py <cpu|cpu-nopeer|gpu|gpu-peer|gpu-flags> <topk|chunk|layer_topk> <d> <steps>      (RANK, WORLD_SIZE, MASTER_* from the env)
 
 Every rank generates all learners' seeded inputs, takes the learner of its own rank through
 multi.LearnerRank, and checks each step's index list, reduced values, its learner's memory and
@@ -12,6 +12,9 @@ another rank, the exchanges are gloo collectives between launches).
 gathered-rows buffers, mapped with CUDA IPC).
 "gpu-flags": as "gpu-peer" without the fence: the reducing kernel waits for flag words the compressing kernels
 set.  Only for a single rank here: kernels of different processes that wait for one another must not share a device.
+"cpu-nopeer": as "cpu", but the ranks ask for the fused exchange (exchange="peer") while a stand-in for the
+device query reports that no rank can reach a peer's memory: every rank must fall back to the collective exchange,
+with a warning, before anything is mapped or stored, and the results stay those of the single-process step.
 "cpu": the same orchestration over an engine made of the oracle's pieces, so that leader rotation,
 broadcast source and row order are checked where there is no GPU.
 """
@@ -81,6 +84,21 @@ def main():
         node = multi.LearnerRank(d, k, beta, lr, layers=layers, exchange=exchange,
                                  selector={"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
                                            "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
+    elif mode == "cpu-nopeer":
+        import warnings
+        asked = []
+
+        def no_access(this_device, peer_device):
+            asked.append((this_device, peer_device))
+            return False
+
+        with warnings.catch_warnings(record=True) as caught:
+            warnings.simplefilter("always")
+            node = multi.LearnerRank(d, k, beta, lr, engine=OracleEngine(d, k, beta, lr, selector, layers), device=dev,
+                                     exchange="peer", can_access_peer=no_access)
+        assert node.exchange == "collective", "the rank kept exchange=%r without peer access" % node.exchange
+        assert any("falls back" in str(c.message) for c in caught), "no warning about the fallback"
+        assert not hasattr(node, "peer_rows"), "buffers were mapped although a peer is out of reach"
     else:
         node = multi.LearnerRank(d, k, beta, lr, engine=OracleEngine(d, k, beta, lr, selector, layers), device=dev)
     prof = workloads.profile(w, dev)

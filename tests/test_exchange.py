@@ -41,6 +41,34 @@ def test_protocol_over_gloo_matches_single_process_step(world, selector):
     run_ranks(world, "cpu", selector, 40_003, 2 * world + 1)
 
 
+def test_fused_exchange_falls_back_when_a_peer_is_out_of_reach():
+    """exchange="peer" stores into other ranks' device memory; when the device query says a peer cannot be reached,
+    all ranks must agree on the collective exchange before anything is mapped (nothing may be stored through an
+    address that was never made accessible)."""
+    run_ranks(2, "cpu-nopeer", "topk", 40_003, 5)
+    run_ranks(3, "cpu-nopeer", "chunk", 20_011, 4)
+
+
+def test_enable_peer_access_checks_its_arguments():
+    """Host-side checks only (no second GPU here): a missing handle is refused."""
+    from paper_2104_11125_b200 import binding
+    assert binding.lib().scalecom_enable_peer_access(None, 0) == binding.ERR_NULL_PTR
+
+
+@pytest.mark.gpu
+def test_enable_peer_access_on_one_device():
+    """With one GPU: the handle's own device needs nothing, an ordinal that does not exist is refused."""
+    import torch
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    with sc.Context(1000, 1, 10, 0.5, 0.1) as ctx:
+        ctx.enable_peer_access(torch.cuda.current_device())
+        for bad in (-1, torch.cuda.device_count()):
+            with pytest.raises(sc.ScaleComError) as e:
+                ctx.enable_peer_access(bad)
+            assert e.value.code == binding.ERR_INVALID_ARG
+
+
 @pytest.mark.gpu
 @pytest.mark.parametrize("world,selector,d", [(2, "topk", 262_147), (3, "topk", 1_048_583), (3, "chunk", 262_147),
                                                 (2, "layer_topk", 262_147)])

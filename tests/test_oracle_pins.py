@@ -461,3 +461,25 @@ def test_layer_topk():
     assert np.array_equal(idx2, oracle.layer_topk(acc[4 % 3].copy(), sizes, keep)[0])
     np.testing.assert_allclose(val, acc[:, idx2].mean(axis=0), rtol=1e-13)
     assert np.array_equal(G, acc[:, idx2])
+
+
+def test_threaded_step_equals_the_plain_step():
+    """The all-cores variant used as the benchmark's parallel CPU baseline hands the plain routines' loops to
+    threads; it must return the same bits (ties at the threshold included, several thread counts, k larger than
+    a thread's range)."""
+    import oracle
+    rng = np.random.default_rng(21)
+    n, d = 5, 50_021
+    g = [rng.standard_normal(d).astype(np.float32) for _ in range(n)]
+    g[2] = (np.round(g[2] * 2) / 2).astype(np.float32)             # heavy ties when learner 2 leads
+    for k in (1, 777, 20_000, d):
+        for threads in (2, 3, 8):
+            m1 = [0.1 * x for x in g]
+            m2 = [x.copy() for x in m1]
+            th1 = np.linspace(-1, 1, d, dtype=np.float32)
+            th2 = th1.copy()
+            for t in range(3):
+                a = oracle.step(g, m1, th1, t, k, 0.25, 0.5)
+                b = oracle.step(g, m2, th2, t, k, 0.25, 0.5, threads=threads)
+                assert all(np.array_equal(x, y) for x, y in zip(a, b)), (k, threads, t)
+            assert all(np.array_equal(x, y) for x, y in zip(m1, m2)) and np.array_equal(th1, th2)
