@@ -31,7 +31,8 @@ MAX_BATCHES = 24                     # distinct gradient batches kept resident; 
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this
 # command with --batches 2) by workload and kernel, with the day of the capture; absent: not captured.
-NCU_TRAFFIC = {"resnet50": {"learner_pass_kernel": 2.4337e9, "topk_select_kernel": 2.167e8, "captured": "2026-11-24"}}
+NCU_TRAFFIC = {"resnet50": {"learner_pass_kernel": 2.4326e9, "topk_select_kernel": 2.205e8, "captured": "2026-11-25"},
+               "resnet50_n16": {"learner_pass_kernel": 4.8896e9, "captured": "2026-11-25"}}
 
 
 def parse_args():
@@ -441,6 +442,7 @@ def bench_workload(args, name, world, rank, dev, stream, barrier, steps=None, la
     ctx.set_option(binding.OPT_KERNEL_SPANS, 0)
     paths = ctx.query(binding.Q_LAST_TOPK_PATH)
     cands = ctx.query(binding.Q_LAST_CANDIDATES)
+    one_kernel = ctx.query(binding.Q_FUSED_SMALL) > 0                  # the whole step is one cooperative kernel
     repeats = []
     for _ in range(args.repeats):
         r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -484,12 +486,26 @@ def bench_workload(args, name, world, rank, dev, stream, barrier, steps=None, la
         peak, peak_src = measured_peak()
         lp_ms = kms[1] / max(ksteps, 1)
         tk_ms = kms[0] / max(ksteps, 1)
-        lp_bytes = 12.0 * w.n * w.d
         tk_bytes = 8.0 * w.d + 4.0 * w.k
+        # the one-kernel step does the selection's reads too: the step's algorithmic bytes are its kernel's
+        lp_bytes = 12.0 * w.n * w.d + (tk_bytes if one_kernel else 0.0)
         lp_gbs = lp_bytes / (lp_ms * 1e-3) / 1e9
-        tk_gbs = tk_bytes / (tk_ms * 1e-3) / 1e9
         traffic = NCU_TRAFFIC.get(w.name, {})
         sel_kernel = {"topk": "topk_select_kernel", "chunk": "chunk_select_kernel", "layer_topk": "layer_topk_kernel"}[args.selector]
+        main_kernel = "small_step_kernel" if one_kernel else "learner_pass_kernel"
+        lp_span = sms[1] / max(ssteps, 1)
+        in_kernel = {"note": "first block start to last block end on the GPU timer, no launch gap or event overhead; "
+                             "same steps as the event figures",
+                     main_kernel: lp_span, "step_frac" if one_kernel else "learner_frac": lp_bytes / (lp_span * 1e-3) / 1e9 / peak}
+        sel_block = None
+        if not one_kernel:
+            tk_gbs = tk_bytes / (tk_ms * 1e-3) / 1e9
+            tk_span = sms[0] / max(ssteps, 1)
+            sel_block = {"achieved": tk_gbs, "frac": tk_gbs / peak, "avg_launch_ms": tk_ms,
+                         "algorithmic_bytes_per_launch": tk_bytes, "traffic": traffic.get(sel_kernel),
+                         "frac_of_nominal_8TBs": tk_gbs / NOMINAL_HBM_GBS}
+            in_kernel[sel_kernel] = tk_span
+            in_kernel["selection_frac"] = tk_bytes / (tk_span * 1e-3) / 1e9 / peak
         out = {
             "metric": METRIC, "value": job_value(w.n, w.d, world, ms_step), "unit": UNIT, "n_gpus": world,
             "steps": K, "warmup": Wm, "ms_per_step": ms_step, "higher_is_better": True,
@@ -503,26 +519,20 @@ def bench_workload(args, name, world, rank, dev, stream, barrier, steps=None, la
                        "gradient_batches_resident": nb, "selector": args.selector,
                        "steps_before_timing": Wm + late_steps,
                        "selection_path_last_step": paths, "selection_candidates_last_step": cands,
+                       "kernels_per_step": 1 if one_kernel else 2,
                        "weight_update": "fused into the learner pass"},
-            "roofline": {"bound": "hbm", "kernel": "learner_pass_kernel", "achieved": lp_gbs, "peak": peak,
-                         "unit": "GB/s", "frac": lp_gbs / peak, "traffic": traffic.get("learner_pass_kernel"),
+            "roofline": {"bound": "hbm", "kernel": main_kernel, "achieved": lp_gbs, "peak": peak,
+                         "unit": "GB/s", "frac": lp_gbs / peak, "traffic": traffic.get(main_kernel),
                          "traffic_captured": traffic.get("captured"),
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": lp_bytes, "avg_launch_ms": lp_ms,
                          "frac_of_nominal_8TBs": lp_gbs / NOMINAL_HBM_GBS,
-                         sel_kernel: {"achieved": tk_gbs, "frac": tk_gbs / peak, "avg_launch_ms": tk_ms,
-                                      "algorithmic_bytes_per_launch": tk_bytes,
-                                      "traffic": traffic.get(sel_kernel),
-                                      "frac_of_nominal_8TBs": tk_gbs / NOMINAL_HBM_GBS},
                          "steps_timed": ksteps, "ms_per_step_with_kernel_events": ms_total_b / K,
-                         "in_kernel_ms": {"note": "first block start to last block end on the GPU timer, no launch "
-                                                  "gap or event overhead; same steps as the event figures",
-                                          "learner_pass_kernel": sms[1] / max(ssteps, 1),
-                                          sel_kernel: sms[0] / max(ssteps, 1),
-                                          "learner_frac": lp_bytes / (sms[1] / max(ssteps, 1) * 1e-3) / 1e9 / peak,
-                                          "selection_frac": tk_bytes / (sms[0] / max(ssteps, 1) * 1e-3) / 1e9 / peak}},
+                         "in_kernel_ms": in_kernel},
             "gpu_launches": launches,
             "clocks": clocks,
         }
+        if sel_block is not None:
+            out["roofline"][sel_kernel] = sel_block
         if repeats:
             rs = sorted(repeats)
             out["repeats"] = {"regions": len(rs), "steps_each": K, "ms_per_step_median": rs[len(rs) // 2],

@@ -255,6 +255,12 @@ int scalecom_reset(scalecom_ctx* ctx);
 #define SCALECOM_OPT_KERNEL_SPANS     7  /* 1: every kernel of a step records the time from its first block's
                                             start to its last block's end on the GPU's nanosecond timer
                                             (two atomics per block); read with scalecom_kernel_span_ms     */
+#define SCALECOM_OPT_FUSED_SMALL      8  /* 1 (default): with the exact top-k selector, at most 8 learners, 16-byte
+                                            aligned vectors and 8*n*d <= 64 MB (all of a step's g and m fit the L2
+                                            cache), scalecom_step runs as ONE cooperative kernel -- selection and
+                                            learner pass share a launch and two grid barriers; 0: always the two
+                                            general kernels.  Affects speed only, never results; per-kernel times
+                                            then report the one kernel in the learner pass's place             */
 #define SCALECOM_SELECTOR_TOPK  0
 #define SCALECOM_SELECTOR_CHUNK 1
 #define SCALECOM_SELECTOR_LAYER_TOPK 2
@@ -269,6 +275,8 @@ int scalecom_set_option(scalecom_ctx* ctx, int option, int64_t value);
 #define SCALECOM_Q_LAST_CANDIDATES  3  /* last step's number of pre-filter survivors                          */
 #define SCALECOM_Q_TOPK_BLOCKS      4  /* thread blocks of the persistent selection kernel                    */
 #define SCALECOM_Q_KERNEL_LAUNCHES  5  /* kernels launched by this handle since creation                      */
+#define SCALECOM_Q_FUSED_SMALL      6  /* thread blocks of the one-kernel step if scalecom_step would use it for
+                                          16-byte aligned vectors (see SCALECOM_OPT_FUSED_SMALL), else 0        */
 #define SCALECOM_Q_PHASE_STAMP0     100 /* +i, i < 13: low 32 bits of the GPU nanosecond timer at phase boundary i of
                                           the last top-k selection kernel (profiling aid): 0-7 as seen by block 0
                                           (start; sample, barrier, bound; filter pass; barrier; k-th key located;

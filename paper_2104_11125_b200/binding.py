@@ -22,10 +22,11 @@ ERR_TIMEOUT, ERR_BAD_STATE, ERR_INTERNAL, ERR_ALIAS = -5, -6, -7, -8
 MAX_LEARNERS = 1024
 
 OPT_FORCE_EXACT_PATH, OPT_SPIN_LIMIT, OPT_KERNEL_TIMING, OPT_FUSE_UPDATE, OPT_USE_HINT, OPT_SELECTOR, OPT_KERNEL_SPANS = 1, 2, 3, 4, 5, 6, 7
+OPT_FUSED_SMALL = 8
 PATH_SAMPLED, PATH_EXACT, PATH_HINTED, PATH_CHUNK, PATH_LAYER_TOPK, PATH_LAYER_TOPK_STREAM = 0, 1, 2, 3, 4, 5
 SELECTOR_TOPK, SELECTOR_CHUNK, SELECTOR_LAYER_TOPK = 0, 1, 2
 Q_PHASE_STAMP0 = 100
-Q_WORKSPACE_BYTES, Q_LAST_TOPK_PATH, Q_LAST_CANDIDATES, Q_TOPK_BLOCKS, Q_KERNEL_LAUNCHES = 1, 2, 3, 4, 5
+Q_WORKSPACE_BYTES, Q_LAST_TOPK_PATH, Q_LAST_CANDIDATES, Q_TOPK_BLOCKS, Q_KERNEL_LAUNCHES, Q_FUSED_SMALL = 1, 2, 3, 4, 5, 6
 
 EXPORTS = (
     "scalecom_create", "scalecom_step", "scalecom_step_host", "scalecom_destroy", "scalecom_set_stream",

@@ -13,7 +13,7 @@ LIB = os.path.join(HERE, "libscalecom.so")
 STAMP = LIB + ".srchash"
 
 SOURCES = ["scalecom.cu", "topk_static.cu"]
-HEADERS = ["common.cuh", "topk_select.cuh", "learner_pass.cuh", "chunk_select.cuh", "diagnostics.cuh", "exchange.cuh", "layer_topk.cuh"]
+HEADERS = ["common.cuh", "topk_select.cuh", "learner_pass.cuh", "chunk_select.cuh", "diagnostics.cuh", "exchange.cuh", "layer_topk.cuh", "small_step.cuh"]
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17",

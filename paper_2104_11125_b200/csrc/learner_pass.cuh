@@ -27,6 +27,7 @@ constexpr int LP_FEW2_BLOCKS_PER_SM = 5;
 constexpr int LP_MID_T = 1;                // 4 to 7 learners: bursts of four learners
 constexpr int LP_MID_BLOCKS_PER_SM = 3;
 constexpr bool LP_MID_EARLY = true;
+constexpr int LP_MANY_BLOCKS_PER_SM = 6;   // 16 learners and more: bursts of one learner
 
 template <int N>
 struct PtrTable {

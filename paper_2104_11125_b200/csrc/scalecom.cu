@@ -14,6 +14,7 @@
 #include "exchange.cuh"
 #include "layer_topk.cuh"
 #include "learner_pass.cuh"
+#include "small_step.cuh"
 #include "topk_select.cuh"
 
 using namespace sc;
@@ -31,6 +32,9 @@ struct scalecom_ctx {
     uint32_t *samp_hist = nullptr, *coarse_win = nullptr, *fine_hist = nullptr, *digit_hist = nullptr;
     uint32_t *ctrl = nullptr, *bitmap = nullptr, *tile_prefix = nullptr, *leader_hint = nullptr;
     uint32_t *block_tot = nullptr;
+    uint32_t *small_tot = nullptr;     // [sms] winners per block of the one-kernel step
+    uint32_t small_blocks = 0;         // its grid, 0: the vector is not eligible (too large, too many learners)
+    bool fused_small = true;           // option: use the one-kernel step where it applies
     uint32_t tiles_per_block = 0;
     mutable uint32_t fine_parity = 0;  // which of the two fine histograms the next top-k launch counts in
     unsigned long long* barrier = nullptr;
@@ -220,13 +224,17 @@ cudaError_t launch_learner(const scalecom_ctx* c, int n, const float* const* gra
 }
 
 // burst shape (tiles x learners) by learner count: few learners take more tiles per burst
-inline int burst_tiles(int n) { return n >= 8 ? 1 : n >= 4 ? 2 : n >= 2 ? 4 : 0; }   // (4 and 0 stand for "2 or 3" and "1")
+inline int burst_tiles(int n) { return n >= 8 ? 1 : n >= 4 ? 2 : n >= 2 ? 4 : 0; }   // (1, 2, 4, 0: "8 or more", "4 to 7", "2 or 3", "1")
 
 template <int N, bool VEC>
 cudaError_t launch_learner_t(const scalecom_ctx* c, int n, const float* const* grads, float* const* mem,
                              const LearnerParams& P) {
     switch (burst_tiles(n)) {
         case 1:
+            // 16 learners and more: one learner per burst at 6 blocks per SM, first burst requested early -- a block
+            // then reads two vectors at a time instead of sixteen, which the DRAM system serves 3-7 % faster once
+            // 32 and more vectors are streamed side by side
+            if (n >= 16) return launch_learner<N, VEC, 1, 1, false, LP_MANY_BLOCKS_PER_SM, true>(c, n, grads, mem, P);
             // 9 to 14 learners: two bursts of equal size instead of eight and the rest
             if (N == 16 && n > 8 && n <= 10) return launch_learner<N, VEC, 1, 5>(c, n, grads, mem, P);
             if (N == 16 && n > 10 && n <= 12) return launch_learner<N, VEC, 1, 6>(c, n, grads, mem, P);
@@ -318,6 +326,36 @@ TopkParams make_topk_params(const scalecom_ctx* c, const float* g, const float* 
     return tp;
 }
 
+// The whole step as one cooperative kernel (vectors whose g and m fit the L2 cache; see small_step.cuh).
+cudaError_t launch_small_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float* weights, int leader,
+                              int32_t* out_idx, float* out_val, unsigned long long* span_slot) {
+    SmallParams P;
+    for (int i = 0; i < SS_MAXN; ++i) {
+        P.tab.g[i] = i < c->n ? grads[i] : nullptr;
+        P.tab.m[i] = i < c->n ? mem[i] : nullptr;
+    }
+    P.d = uint32_t(c->d); P.k = uint32_t(c->k); P.ntiles = c->ntiles;
+    P.n = c->n; P.leader = leader;
+    P.beta = c->beta; P.omb = 1.0f - c->beta; P.lr = c->lr; P.nf = float(c->n);
+    P.force_exact = c->force_exact; P.use_hint = c->use_hint; P.spin_limit = c->spin_limit;
+    P.leader_hint = c->leader_hint + leader; P.all_hints = c->leader_hint; P.n_hints = uint32_t(c->n);
+    P.key_hist = c->samp_hist; P.coarse_win = c->coarse_win;
+    P.fine_hist = c->fine_hist + size_t(c->fine_parity) * NFINE;
+    P.fine_hist_next = c->fine_hist + size_t(c->fine_parity ^ 1u) * NFINE;
+    c->fine_parity ^= 1u;
+    P.digit_hist = c->digit_hist; P.block_tot = c->small_tot; P.ctrl = c->ctrl;
+    P.barrier = c->barrier + 24;               // its own arrival counter: its grid differs from the other kernels'
+    P.blist = c->blist;
+    P.out_idx = out_idx; P.out_val = out_val; P.gathered = c->gathered;
+    P.weights = (weights && c->fuse_update) ? weights : nullptr;
+    P.spans = span_slot;
+    c->bitmap_zero = false;
+    c->select_fresh = false;
+    void* args[] = {&P};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(&small_step_kernel), dim3(c->small_blocks),
+                                       dim3(SS_THREADS), args, sizeof(SmallShared), c->stream);
+}
+
 int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float* weights, int64_t t, int32_t* out_idx,
             float* out_val) {
     const int leader = int(t % c->n);
@@ -361,6 +399,29 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
     cudaEvent_t* ev = tm ? c->ev + 4 * (c->ev_steps % scalecom_ctx::EV_RING) : nullptr;
     if (tm && cudaEventRecord(ev[0], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
     cudaError_t e;
+    if (c->small_blocks && c->fused_small && vec_all && c->selector == SCALECOM_SELECTOR_TOPK) {
+        // one kernel for the whole step; in the per-kernel figures it takes the learner pass's place and the
+        // selection's interval is empty
+        if (tm && cudaEventRecord(ev[1], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+        e = launch_small_step(c, grads, mem, weights, leader, out_idx, out_val, span_slot ? span_slot + 2 : nullptr);
+        if (e != cudaSuccess) { cudaGetLastError(); return SCALECOM_ERR_CUDA; }
+        ++c->launches;
+        if (tm && cudaEventRecord(ev[2], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+        if (weights && !c->fuse_update) {
+            const uint32_t blocks = uint32_t((c->k + 255) / 256);
+            apply_update_kernel<<<blocks < 4096u ? blocks : 4096u, 256, 0, c->stream>>>(weights, out_idx, out_val,
+                                                                                       uint32_t(c->k), c->lr, c->ctrl + CT_STATUS);
+            if (cudaGetLastError() != cudaSuccess) return SCALECOM_ERR_CUDA;
+            ++c->launches;
+        }
+        if (tm) {
+            c->ev_has_update[c->ev_steps % scalecom_ctx::EV_RING] = weights && !c->fuse_update;
+            if (weights && !c->fuse_update && cudaEventRecord(ev[3], c->stream) != cudaSuccess) return SCALECOM_ERR_CUDA;
+            ++c->ev_steps;
+        }
+        if (span_slot) ++c->span_steps;
+        return SCALECOM_OK;
+    }
     if (c->selector == SCALECOM_SELECTOR_CHUNK) {
         ChunkParams cp;
         cp.g = tp.g; cp.m = tp.m; cp.d = tp.d; cp.k = tp.k;
@@ -450,6 +511,19 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     if (c->topk_blocks > chunks) c->topk_blocks = chunks;
     if (c->topk_blocks < 1) c->topk_blocks = 1;
     c->tiles_per_block = (c->ntiles + c->topk_blocks - 1) / c->topk_blocks;
+    {
+        // the one-kernel step: at most SS_MAXN learners, a block's share of the tiles within its shared-memory
+        // bitmap, and all g and m of a step (8 n d bytes) within 64 MB, about half the L2 cache
+        int occ_small = 0;
+        const bool fits = n <= SS_MAXN && uint64_t(c->ntiles) <= uint64_t(SS_TILES) * uint64_t(c->sms) &&
+                          uint64_t(n) * uint64_t(d) <= (1ull << 23);
+        if (fits &&
+            cudaFuncSetAttribute(small_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(sizeof(SmallShared))) == cudaSuccess &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_small, small_step_kernel, SS_THREADS, sizeof(SmallShared)) == cudaSuccess &&
+            occ_small >= 1)
+            c->small_blocks = c->ntiles < uint32_t(c->sms) ? c->ntiles : uint32_t(c->sms);
+        cudaGetLastError();
+    }
     c->lp_blocks = uint32_t(c->sms * occ_lp);
     if (c->lp_blocks > c->ntiles) c->lp_blocks = c->ntiles;
 
@@ -484,7 +558,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     size_t off = 0;
     auto carve = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
     const size_t o_samp = carve(NCOARSE * 4), o_cw = carve((WIN + 1) * 4), o_ctrl = carve(CT_WORDS * 4), o_bar = carve(256);
-    const size_t o_lh = carve(size_t(n) * 4), o_bt = carve(size_t(c->topk_blocks) * 4);
+    const size_t o_lh = carve(size_t(n) * 4), o_bt = carve(size_t(c->topk_blocks) * 4), o_st = carve(size_t(c->sms) * 4);
     const size_t o_fine = carve(2 * size_t(NFINE) * 4), o_dh = carve(size_t(DH_PASSES) * DH_BINS * 4);
     c->ctrl_region_bytes = off;                 // everything the kernel expects to find zero
     const size_t o_cand = carve(size_t(c->seg_cap) * c->topk_blocks * TK_WARPS * 8), o_bl = carve(size_t(BCAP) * 8);
@@ -501,6 +575,7 @@ int scalecom_create(scalecom_ctx** out, int64_t d, int32_t n, int64_t k, float b
     c->ctrl = reinterpret_cast<uint32_t*>(base + o_ctrl);
     c->barrier = reinterpret_cast<unsigned long long*>(base + o_bar);
     c->block_tot = reinterpret_cast<uint32_t*>(base + o_bt);
+    c->small_tot = reinterpret_cast<uint32_t*>(base + o_st);
     c->leader_hint = reinterpret_cast<uint32_t*>(base + o_lh);
     c->fine_hist = reinterpret_cast<uint32_t*>(base + o_fine);
     c->digit_hist = reinterpret_cast<uint32_t*>(base + o_dh);
@@ -861,6 +936,7 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
         }
         case SCALECOM_OPT_FUSE_UPDATE: c->fuse_update = value != 0; return SCALECOM_OK;
         case SCALECOM_OPT_USE_HINT: c->use_hint = value ? 1u : 0u; return SCALECOM_OK;
+        case SCALECOM_OPT_FUSED_SMALL: c->fused_small = value != 0; return SCALECOM_OK;
         case SCALECOM_OPT_KERNEL_SPANS: {
             DeviceGuard guard(c->device);
             const size_t bytes = size_t(scalecom_ctx::EV_RING) * 4 * 8;
@@ -931,6 +1007,9 @@ int scalecom_query(scalecom_ctx* c, int item, int64_t* out) {
             return SCALECOM_OK;
         case SCALECOM_Q_TOPK_BLOCKS: *out = c->topk_blocks; return SCALECOM_OK;
         case SCALECOM_Q_KERNEL_LAUNCHES: *out = c->launches; return SCALECOM_OK;
+        case SCALECOM_Q_FUSED_SMALL:
+            *out = (c->small_blocks && c->fused_small && c->selector == SCALECOM_SELECTOR_TOPK) ? c->small_blocks : 0;
+            return SCALECOM_OK;
         case SCALECOM_Q_LAST_TOPK_PATH:
         case SCALECOM_Q_LAST_CANDIDATES:
             if (cudaStreamSynchronize(c->stream) != cudaSuccess ||

@@ -114,7 +114,9 @@ struct TopkShared {
 // Block-wide search from the top of a histogram of nb <= TK_THREADS bins held one bin per thread: thread r holds
 // v = h[nb - 1 - r] (0 for r >= nb).  Finds the bin holding the `need`-th element counted from the top:
 // s.res = {bin, count strictly above bin, count in bin}, bin = 0xFFFFFFFF when the histogram holds fewer.
-__device__ inline void find_in_regs(uint32_t v, uint32_t nb, uint32_t need, TopkShared& s) {
+// (Shared: any shared-memory struct with scan[32] and res[4].)
+template <class Shared>
+__device__ inline void find_in_regs(uint32_t v, uint32_t nb, uint32_t need, Shared& s) {
     const uint32_t lane = lane_id(), warp = warp_id(), r = threadIdx.x;
     if (threadIdx.x == 0) s.res[0] = 0xFFFFFFFFu;
     const uint32_t incl = warp_incl_scan(v);
@@ -130,7 +132,8 @@ __device__ inline void find_in_regs(uint32_t v, uint32_t nb, uint32_t need, Topk
 
 // The same for a histogram in global memory (written by other blocks before the last grid barrier) of up to 8192
 // bins: TK_WARPS warp-sized segments first, then one bin per thread inside the segment that holds the answer.
-__device__ inline void find_from_top(const uint32_t* h, uint32_t nb, uint32_t need, TopkShared& s) {
+template <class Shared>
+__device__ inline void find_from_top(const uint32_t* h, uint32_t nb, uint32_t need, Shared& s) {
     const uint32_t lane = lane_id(), warp = warp_id();
     if (nb <= uint32_t(TK_THREADS)) {
         const uint32_t r = threadIdx.x;

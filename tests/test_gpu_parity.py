@@ -157,7 +157,7 @@ def test_host_buffer_entry_point():
     assert np.array_equal(th.cpu().numpy(), th_o)
 
 
-@pytest.mark.parametrize("selector", ["topk", "chunk", "layer_topk"])
+@pytest.mark.parametrize("selector", ["topk", "topk-two-kernels", "chunk", "layer_topk"])
 def test_bounded_wait_expiry_is_reported_and_recoverable(selector):
     """Failure detection without a GPU fault: with the barrier's iteration bound set to 0 every
     wait gives up at once, the kernel returns, the status word says TIMEOUT, the kernels that follow it in
@@ -166,7 +166,9 @@ def test_bounded_wait_expiry_is_reported_and_recoverable(selector):
     import oracle
     import paper_2104_11125_b200 as sc
     from paper_2104_11125_b200 import binding
-    w = W.TINY.scaled(200_000)                      # 25 blocks in the selection kernel
+    w = W.TINY.scaled(200_000)                      # 25 blocks in the selection kernel, 148 in the one-kernel step
+    two_kernels = selector == "topk-two-kernels"    # "topk" alone: the one-kernel step this size takes by default
+    selector = "topk" if two_kernels else selector
     prof = W.profile(w, DEV)
     g = W.gradients(w, 0, DEV, prof)
     idx = torch.full((w.k,), -7, device=DEV, dtype=torch.int32)
@@ -178,6 +180,8 @@ def test_bounded_wait_expiry_is_reported_and_recoverable(selector):
                                               "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
         if layers:
             ctx.set_layers(*layers)
+        ctx.set_option(binding.OPT_FUSED_SMALL, 0 if two_kernels else 1)
+        assert (ctx.query(binding.Q_FUSED_SMALL) > 0) == (selector == "topk" and not two_kernels)
         ctx.set_option(binding.OPT_SPIN_LIMIT, 0)
         m = [torch.full((w.d,), 0.25, device=DEV) for _ in range(w.n)]
         theta = torch.full((w.d,), 1.5, device=DEV)
@@ -302,8 +306,10 @@ def test_switching_selectors_on_one_handle():
         assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(m, m_o))
 
 
-def test_kernel_timing_queries():
-    """Per-kernel CUDA-event times and in-kernel time spans: positive, consistent, reset on read."""
+@pytest.mark.parametrize("fused", [False, True])
+def test_kernel_timing_queries(fused):
+    """Per-kernel CUDA-event times and in-kernel time spans: positive, consistent, reset on read.  With the
+    one-kernel step the whole step is reported in the learner pass's place and the selection's interval is empty."""
     import paper_2104_11125_b200 as sc
     from paper_2104_11125_b200 import binding
     w = W.TINY.scaled(1_000_000)
@@ -314,14 +320,22 @@ def test_kernel_timing_queries():
     with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
         with pytest.raises(sc.ScaleComError):
             ctx.kernel_span_ms()                       # option off
+        ctx.set_option(binding.OPT_FUSED_SMALL, int(fused))
+        assert (ctx.query(binding.Q_FUSED_SMALL) > 0) == fused
         ctx.set_option(binding.OPT_KERNEL_TIMING, 1)
         ctx.set_option(binding.OPT_KERNEL_SPANS, 1)
+        launches0 = ctx.query(binding.Q_KERNEL_LAUNCHES)
         for t in range(5):
             ctx.step(W.gradients(w, t, DEV, prof), m, None, t, idx, val)
+        assert ctx.query(binding.Q_KERNEL_LAUNCHES) - launches0 == (5 if fused else 10)
         ev, ne = ctx.kernel_ms()
         sp, ns = ctx.kernel_span_ms()
         assert ne == 5 and ns == 5
-        assert 0 < sp[0] <= ev[0] * 1.05 and 0 < sp[1] <= ev[1] * 1.05     # a span lies inside its event interval
+        if fused:
+            assert sp[0] == 0.0 and ev[0] < 0.25 * ev[1]                     # nothing runs in the selection's interval
+        else:
+            assert 0 < sp[0] <= ev[0] * 1.05                                 # a span lies inside its event interval
+        assert 0 < sp[1] <= ev[1] * 1.05
         assert ev[2] == 0.0                                                  # weight update fused: no third kernel
         assert ctx.kernel_ms()[1] == 0 and ctx.kernel_span_ms()[1] == 0      # both forget what they reported
         assert ctx.status() == 0
