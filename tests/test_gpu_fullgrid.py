@@ -9,7 +9,7 @@ compared element by element with the oracle's step:
     candidate segments, down to the index digits;
   * vectors on which the pre-filter cannot work at all (all coordinates equal; nine tenths zero
     with k beyond the non-zeros): the exact route, every pass streaming g and m again;
-  * config 2 for 20 steps from a cold start with the window method of test_gpu_fullsize.py,
+  * config 2 for 16 steps from a cold start with the window method of test_gpu_fullsize.py,
     recording which route every step took.
 """
 import numpy as np
@@ -98,12 +98,12 @@ def test_exact_route_at_full_grid():
     assert paths[0] == binding.PATH_SAMPLED, paths
 
 
-def test_config2_twenty_steps_route_mix():
-    """Config 2 at full size for 20 steps (every learner leads at least twice): selection in full and the
+def test_config2_sixteen_steps_route_mix():
+    """Config 2 at full size for 16 steps (every learner leads twice): selection in full and the
     other outputs inside windows, every step; the routes taken are asserted as a mix, not step by step."""
     from paper_2104_11125_b200 import binding
     from tests.test_gpu_fullsize import fullsize_case
-    paths = fullsize_case(W.RESNET50, steps=20, strict_paths=False)
+    paths = fullsize_case(W.RESNET50, steps=16, strict_paths=False)
     assert paths[0] == binding.PATH_SAMPLED
     assert all(p in (binding.PATH_SAMPLED, binding.PATH_HINTED) for p in paths), paths
-    assert paths.count(binding.PATH_HINTED) >= 16, paths           # the hint carries almost every step
+    assert paths.count(binding.PATH_HINTED) >= 13, paths           # the hint carries almost every step
