@@ -635,3 +635,39 @@ def test_drifting_scale_run_stays_exact_and_mostly_hinted():
                 assert all(np.array_equal(a.cpu().numpy(), b) for a, b in zip(mem, m_o)), t
                 assert np.array_equal(theta.cpu().numpy(), th_o), t
     assert sampled <= 60, sampled
+
+
+# ---- the one-kernel step at the edges of what it accepts --------------------------------------------------
+def test_one_kernel_step_at_its_largest_ranges_and_on_its_fallbacks():
+    """The one-kernel step (small vectors) with as many tiles per block as it takes (14 and 16 of 16), with all of
+    the top-k inside one block's range (its shared-memory survivor list overflows: radix select over the range),
+    and with more equal keys around rank k than the boundary list holds.  run_and_compare runs each case with the
+    kernel and with the two general kernels."""
+    import paper_2104_11125_b200 as sc
+    from paper_2104_11125_b200 import binding
+    p = _parity()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for d, n in ((2_000_003, 2), (16 * 1024 * sms - 5, 3)):
+        w = W.TINY.scaled(d, n=n)
+        with sc.Context(w.d, w.n, w.k, w.beta, w.lr) as ctx:
+            assert ctx.query(binding.Q_FUSED_SMALL) == sms, "the case is not taken by the one-kernel step"
+        p.workload_case(w, 3, DEV, want_path=0)
+    rng = np.random.default_rng(31)
+    d, k = 1_000_003, 9000
+    theta = torch.linspace(-1, 1, d, device=DEV)
+    m0 = [torch.zeros(d, device=DEV) for _ in range(2)]
+    # every large coordinate inside 9000 consecutive ones: one block finds them all
+    x = (1e-3 * rng.standard_normal(d)).astype(np.float32)
+    x[500_000:500_000 + 12_000] = rng.standard_normal(12_000).astype(np.float32)
+    g = [torch.tensor(x, device=DEV), torch.tensor(0.5 * x, device=DEV)]
+    paths = p.run_and_compare([g, g, g], m0, theta, k, 0.5, 0.25, tag="clustered", fused_small=True)
+    assert binding.PATH_EXACT in paths, paths
+    # 3000 copies of the k-th magnitude: beyond the 1024-entry boundary list
+    y = rng.standard_normal(d).astype(np.float32)
+    tau = np.sort(np.abs(y))[-k]
+    ties = rng.choice(d, 3000, replace=False)
+    y[ties] = np.where(rng.random(3000) < 0.5, tau, -tau).astype(np.float32)
+    g = [torch.tensor(y, device=DEV), torch.tensor(-0.25 * y, device=DEV)]
+    paths = p.run_and_compare([g, g], m0, theta, k, 0.5, 0.25, tag="3000-ties", fused_small=True)
+    assert binding.PATH_EXACT in paths, paths
+    p.run_and_compare([g, g], m0, theta, k, 0.5, 0.25, tag="3000-ties", fused_small=False)
