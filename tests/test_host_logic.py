@@ -122,6 +122,25 @@ def test_bench_reference_arm_prints_the_contract_line():
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["steps"] == 2
 
 
+def test_bench_reference_arm_keeps_the_workload_and_names_its_sample():
+    """The reference arm reports the workload's own n, d, k (so that the two arms' configurations can be compared)
+    and says in cpu_baseline.sample whether it ran whole steps or a bounded part of every vector."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert (line["config"]["n"], line["config"]["d"], line["config"]["k"]) == (4, 1 << 20, 10485)
+    assert line["cpu_baseline"]["sample"].startswith("full steps of the workload")
+
+
+def test_learner_sweep_fit_is_a_least_squares_line():
+    import bench
+    slope, icpt = bench.fit_line([8, 32, 64, 128], [0.05 * n + 0.07 for n in (8, 32, 64, 128)])
+    assert abs(slope - 0.05) < 1e-12 and abs(icpt - 0.07) < 1e-12
+    slope, icpt = bench.fit_line([1, 2, 3], [1.0, 2.0, 4.0])
+    assert abs(slope - 1.5) < 1e-12 and abs(icpt - (7.0 / 3 - 3.0)) < 1e-12
+
+
 _GLOO_WORKER = r"""
 import os, sys
 sys.path.insert(0, sys.argv[1])
