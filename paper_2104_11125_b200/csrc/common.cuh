@@ -45,6 +45,14 @@ __device__ __forceinline__ void load_quad_stream(const float* __restrict__ a, ui
     }
 }
 
+// 128-bit load with an L2 cache-hint policy (createpolicy); p is 16-byte aligned
+__device__ __forceinline__ float4 ld_quad_policy(const float* p, uint64_t policy) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(policy));
+    return v;
+}
+
 template <bool VEC>
 __device__ __forceinline__ void store_quad_stream(float* __restrict__ a, uint32_t p, uint32_t d, const float (&v)[4]) {
     if (VEC && p + 4u <= d) {

@@ -58,6 +58,8 @@ constexpr uint32_t DH_BINS = 2048;                             // digit histogra
 constexpr uint32_t DH_PASSES = 8;
 constexpr uint32_t SAMPLE_GRANULE = 128;                       // coordinates one warp samples at a time
 constexpr uint32_t BCAP = 1024;                                // boundary list entries
+constexpr double KEEP_SHARE = 0.25;                            // largest share of the leader's lines held in L2 for the learner pass
+constexpr double KEEP_SHARE_MIN = 0.05;                        // and the smallest worth marking the stream for
 
 // ctrl words
 constexpr int CT_CAND = 0, CT_STATUS = 1, CT_PATH = 2, CT_M = 3, CT_BCOUNT = 4, CT_OVERFLOW = 5, CT_HINT = 6, CT_MARGIN = 7;
@@ -79,6 +81,7 @@ struct TopkParams {
     uint32_t* all_hints;       // every leader's entry [n_hints] (or nullptr): forgotten when a hint turns out useless
     uint32_t n_hints;
     uint32_t spin_limit;
+    float keep_frac;           // share of the leader's lines asked to stay in L2 for the kernel that reads them next (0: none)
     // the four histograms are all zero on entry and all zero again on exit
     uint32_t* samp_hist;       // [NCOARSE]
     uint32_t* coarse_win;      // [WIN + 1]
@@ -354,6 +357,14 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                 bal = __ballot_sync(FULL, nib != 0);
             }
         };
+        // L2 policy of the stream: a share of the lines is marked to be replaced last, so that the learner pass, which
+        // reads the leader's g and m once more, finds them in the cache; the rest is marked to be replaced first and
+        // recycles itself instead of pushing out what the previous kernel left there.
+        uint64_t stream_policy;
+        if (P.keep_frac > 0.0f)
+            asm volatile("createpolicy.fractional.L2::evict_last.L2::evict_first.b64 %0, %1;" : "=l"(stream_policy) : "f"(P.keep_frac));
+        else
+            asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(stream_policy));
         for (uint32_t it0 = 0; it0 < my_units; it0 += TK_UNROLL) {
             float gv[TK_UNROLL][4], mv[TK_UNROLL][4];
             const bool whole = VEC && it0 + TK_UNROLL <= my_units &&
@@ -363,8 +374,8 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
 #pragma unroll
                 for (int u = 0; u < TK_UNROLL; ++u) {
                     const uint32_t p = pbase + u * (nblocks * TK_UNIT);
-                    const float4 a = *reinterpret_cast<const float4*>(P.g + p);
-                    const float4 b = *reinterpret_cast<const float4*>(P.m + p);
+                    const float4 a = ld_quad_policy(P.g + p, stream_policy);
+                    const float4 b = ld_quad_policy(P.m + p, stream_policy);
                     gv[u][0] = a.x; gv[u][1] = a.y; gv[u][2] = a.z; gv[u][3] = a.w;
                     mv[u][0] = b.x; mv[u][1] = b.y; mv[u][2] = b.z; mv[u][3] = b.w;
                 }

@@ -126,6 +126,7 @@ extern "C" int scalecom_topk_static(const float* g, const float* m, int64_t d, i
         }
     }
     P.force_exact = 0;
+    P.keep_frac = 0.0f;
     P.use_hint = 0;               // the scratch is shared by unrelated callers: no carry-over between calls
     P.leader_hint = nullptr;
     P.all_hints = nullptr;
