@@ -49,7 +49,7 @@ __device__ __forceinline__ void load_quad_stream(const float* __restrict__ a, ui
 __device__ __forceinline__ float4 ld_quad_policy(const float* p, uint64_t policy) {
     float4 v;
     asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(policy));
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(__cvta_generic_to_global(p)), "l"(policy));
     return v;
 }
 
