@@ -261,6 +261,13 @@ int scalecom_reset(scalecom_ctx* ctx);
                                             learner pass share a launch and two grid barriers; 0: always the two
                                             general kernels.  Affects speed only, never results; per-kernel times
                                             then report the one kernel in the learner pass's place             */
+#define SCALECOM_OPT_L2_KEEP          9  /* 1 (default): the exact top-k selection of scalecom_step loads a share of
+                                            the leader's g and m (a quarter of the lines, at most 0.4 of the L2
+                                            cache; none for vectors of which the cache holds under a twentieth) with
+                                            a replace-last L2 hint and the rest with a replace-first hint, because
+                                            the learner pass reads both vectors again.  The marked lines keep their
+                                            priority until something replaces them; 0: default L2 policy.  Affects
+                                            speed only, never results                                            */
 #define SCALECOM_SELECTOR_TOPK  0
 #define SCALECOM_SELECTOR_CHUNK 1
 #define SCALECOM_SELECTOR_LAYER_TOPK 2

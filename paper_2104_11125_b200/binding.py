@@ -23,6 +23,7 @@ MAX_LEARNERS = 1024
 
 OPT_FORCE_EXACT_PATH, OPT_SPIN_LIMIT, OPT_KERNEL_TIMING, OPT_FUSE_UPDATE, OPT_USE_HINT, OPT_SELECTOR, OPT_KERNEL_SPANS = 1, 2, 3, 4, 5, 6, 7
 OPT_FUSED_SMALL = 8
+OPT_L2_KEEP = 9
 PATH_SAMPLED, PATH_EXACT, PATH_HINTED, PATH_CHUNK, PATH_LAYER_TOPK, PATH_LAYER_TOPK_STREAM = 0, 1, 2, 3, 4, 5
 SELECTOR_TOPK, SELECTOR_CHUNK, SELECTOR_LAYER_TOPK = 0, 1, 2
 Q_PHASE_STAMP0 = 100

@@ -50,6 +50,7 @@ struct scalecom_ctx {
     mutable bool bitmap_zero = false;  // the bitmap holds no bits (scalecom_compress leaves it so; selection kernels do not)
     uint32_t samp_stride = 1, samp_target = 1;
     float keep_frac = 0.0f;            // share of the leader's lines a step's selection asks L2 to hold for the learner pass
+    bool l2_keep = true;               // SCALECOM_OPT_L2_KEEP
 
     // options
     uint32_t force_exact = 0;
@@ -374,7 +375,7 @@ int do_step(scalecom_ctx* c, const float* const* grads, float* const* mem, float
         cudaMemsetAsync(span_slot, 0, 4 * sizeof(unsigned long long), c->stream) != cudaSuccess)
         return SCALECOM_ERR_CUDA;
     TopkParams tp = make_topk_params(c, grads[leader], mem[leader], c->leader_hint + leader, true, span_slot);
-    tp.keep_frac = c->keep_frac;
+    tp.keep_frac = c->l2_keep ? c->keep_frac : 0.0f;
 
     LearnerParams lp;
     lp.d = uint32_t(c->d);
@@ -951,6 +952,7 @@ int scalecom_set_option(scalecom_ctx* c, int option, int64_t value) {
         case SCALECOM_OPT_FUSE_UPDATE: c->fuse_update = value != 0; return SCALECOM_OK;
         case SCALECOM_OPT_USE_HINT: c->use_hint = value ? 1u : 0u; return SCALECOM_OK;
         case SCALECOM_OPT_FUSED_SMALL: c->fused_small = value != 0; return SCALECOM_OK;
+        case SCALECOM_OPT_L2_KEEP: c->l2_keep = value != 0; return SCALECOM_OK;
         case SCALECOM_OPT_KERNEL_SPANS: {
             DeviceGuard guard(c->device);
             const size_t bytes = size_t(scalecom_ctx::EV_RING) * 4 * 8;

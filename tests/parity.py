@@ -42,20 +42,22 @@ def assert_step_matches(tag, idx_g, val_g, G_g, m_g, th_g, idx_o, val_o, G_o, m_
 
 
 def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exact=False, fuse_update=True,
-                    want_path=None, offset=0, use_hint=True, selector="topk", layers=None, tag="case", fused_small=None):
+                    want_path=None, offset=0, use_hint=True, selector="topk", layers=None, tag="case", fused_small=None,
+                    l2_keep=True):
     """grads_per_step: list over steps of lists of n CUDA fp32 tensors.
     m0: list of n CUDA tensors (initial memory), theta0: CUDA tensor or None.
     offset > 0 places every device vector `offset` floats past a 16-byte boundary
     (exercises the unaligned code path).
     fused_small: True / False pins whether small vectors take the one-kernel step; None (default) runs the case
-    both ways when the library would use that kernel for it, and returns the paths of the two-kernel run."""
+    both ways when the library would use that kernel for it, and returns the paths of the two-kernel run.
+    l2_keep: SCALECOM_OPT_L2_KEEP (speed only: results must not depend on it)."""
     dev = grads_per_step[0][0].device
     n, d = len(m0), m0[0].numel()
     if fused_small is None:
         with sc.Context(d, n, k, beta, lr) as probe:
             eligible = probe.query(binding.Q_FUSED_SMALL) > 0 and selector == "topk" and offset % 4 == 0
         kw = dict(force_exact=force_exact, fuse_update=fuse_update, want_path=want_path, offset=offset, use_hint=use_hint,
-                  selector=selector, layers=layers)
+                  selector=selector, layers=layers, l2_keep=l2_keep)
         if eligible:
             run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0, tag=tag + " (one kernel)", fused_small=True, **kw)
         return run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0, tag=tag, fused_small=False, **kw)
@@ -82,6 +84,7 @@ def run_and_compare(grads_per_step, m0, theta0, k, beta, lr, t0=0, *, force_exac
         ctx.set_option(binding.OPT_FUSE_UPDATE, int(fuse_update))
         ctx.set_option(binding.OPT_USE_HINT, int(use_hint))
         ctx.set_option(binding.OPT_FUSED_SMALL, int(fused_small))
+        ctx.set_option(binding.OPT_L2_KEEP, int(l2_keep))
         ctx.set_option(binding.OPT_SELECTOR, {"topk": binding.SELECTOR_TOPK, "chunk": binding.SELECTOR_CHUNK,
                                               "layer_topk": binding.SELECTOR_LAYER_TOPK}[selector])
         if layers is not None:

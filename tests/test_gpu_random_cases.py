@@ -61,4 +61,5 @@ def test_random_cases_match_the_oracle(seed):
         theta0 = torch.linspace(-1, 1, c["d"], device=DEV)
         p.run_and_compare(grads, m0, theta0, c["k"], c["beta"], 0.25, t0=c["t0"], force_exact=c["force_exact"],
                           fuse_update=c["fuse_update"], offset=c["offset"], use_hint=c["use_hint"],
-                          selector=c["selector"], layers=c["layers"], tag=tag)
+                          selector=c["selector"], layers=c["layers"], tag=tag,
+                          l2_keep=(c["d"] + c["n"] + c["k"]) % 3 != 0)      # (derived, so that the drawn cases stay the same)

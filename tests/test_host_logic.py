@@ -32,6 +32,18 @@ def test_library_exports_every_declared_symbol(lib):
         assert getattr(lib, name) is not None
 
 
+def test_binding_constants_equal_the_header_defines():
+    """Every SCALECOM_OPT_ / _Q_ / _SELECTOR_ define of the header has a constant of the same value in the binding."""
+    from paper_2104_11125_b200 import binding
+    header = open(os.path.join(ROOT, "include", "scalecom.h")).read()
+    defines = re.findall(r"#define\s+SCALECOM_((?:OPT|Q|SELECTOR)_[A-Z0-9_]+)\s+(-?\d+)", header)
+    defines += re.findall(r"SCALECOM_(OK|ERR_[A-Z_]+)\s*=\s*(-?\d+)", header)      # the error enum
+    assert len(defines) >= 28
+    for name, value in defines:
+        assert hasattr(binding, name), "binding lacks %s" % name
+        assert getattr(binding, name) == int(value), name
+
+
 def test_create_rejects_bad_arguments_without_touching_the_gpu(lib):
     from paper_2104_11125_b200 import binding as b
     bad = [
