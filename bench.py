@@ -67,6 +67,8 @@ def parse_args():
                          "compressing kernel as stores into the peers' mapped buffers, a one-word all-reduce as fence "
                          "(peer); or the same with flag words the reducing kernel waits for instead of the fence "
                          "(peer-flags; one rank per GPU)")
+    ap.add_argument("--l2-keep", type=int, default=1, choices=[0, 1],
+                    help="SCALECOM_OPT_L2_KEEP: 0 streams the leader's vectors with the default L2 policy (for A/B runs and captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -399,6 +401,8 @@ def bench_workload(args, name, world, rank, dev, stream, barrier, steps=None, la
         ctx.set_option(binding.OPT_SELECTOR, binding.SELECTOR_CHUNK)
     if layers is not None:
         ctx.set_layers(*layers)
+    if not args.l2_keep:
+        ctx.set_option(binding.OPT_L2_KEEP, 0)
     torch.cuda.synchronize()
     step = ctx.prepare_step(batches, mem, theta, idx, val)        # pointer tables marshalled once per batch
 
@@ -516,7 +520,7 @@ def bench_workload(args, name, world, rank, dev, stream, barrier, steps=None, la
                              if 8 * w.n * w.d > 126e6 else
                              "g+m (%.0f MB) fit L2: the memories stay cached from step to step, the gradients cycle through "
                              "%d resident batches (%.0f MB) and come from HBM" % (8e-6 * w.n * w.d, nb, 4e-6 * nb * w.n * w.d),
-                       "gradient_batches_resident": nb, "selector": args.selector,
+                       "gradient_batches_resident": nb, "selector": args.selector, "l2_keep": args.l2_keep,
                        "steps_before_timing": Wm + late_steps,
                        "selection_path_last_step": paths, "selection_candidates_last_step": cands,
                        "kernels_per_step": 1 if one_kernel else 2,
