@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(LP_THREADS, MINB)
 learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams P, const __grid_constant__ PeerTable peers) {
     static_assert(LP_T * LP_L <= LP_UNROLL, "burst shape");
     constexpr bool GUARD = ONE;
+    constexpr bool TAIL_LOOP = LP_L >= 5;
     const uint32_t tid = threadIdx.x, lane = lane_id();
     const uint32_t d = P.d;
     const int n = N1 ? 1 : P.n;                    // N1: one learner, known when compiling
@@ -176,17 +177,36 @@ learner_pass_kernel(const __grid_constant__ PtrTable<N> tab, const LearnerParams
         for (int t = 0; t < LP_T; ++t)
             if (nib[t] && pc[t] < d) {
                 uint32_t r = rank0[t];
+                if (!TAIL_LOOP) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (((nib[t] >> c) & 1u) && (!GUARD || r < P.k)) {
-                        const float v = __fdiv_rn(sum[t][c], P.nf);                           // line 10: one division by n
-                        P.out_idx[r] = int32_t(pc[t] + c);
-                        P.out_val[r] = v;
-                        if (ONE)
-                            for (int q = 0; q < peers.n; ++q) peers.dst[q][r] = v;    // Eq. 3's values, sent as they are made
-                        ++r;
-                        if (weights) weights[pc[t] + c] = __fsub_rn(wv[t][c], __fmul_rn(P.lr, v));   // line 12
-                    }
+                    for (int c = 0; c < 4; ++c)
+                        if (((nib[t] >> c) & 1u) && (!GUARD || r < P.k)) {
+                            const float v = __fdiv_rn(sum[t][c], P.nf);                       // line 10: one division by n
+                            P.out_idx[r] = int32_t(pc[t] + c);
+                            P.out_val[r] = v;
+                            if (ONE)
+                                for (int q = 0; q < peers.n; ++q) peers.dst[q][r] = v;    // Eq. 3's values, sent as they are made
+                            ++r;
+                            if (weights) weights[pc[t] + c] = __fsub_rn(wv[t][c], __fmul_rn(P.lr, v));   // line 12
+                        }
+                    continue;
+                }
+                // bursts of five learners and more: one turn per selected coordinate of the lane (usually one), so that
+                // the division is not laid out four times (8 learners: -1 us; evenly spread picks, as the chunk-wise
+                // selector and a long run leave them: -2 to -4 us; the shapes for fewer learners measured slower with it)
+                for (uint32_t left = nib[t]; left; left &= left - 1u) {
+                    const uint32_t c = __ffs(left) - 1u;
+                    if (GUARD && r >= P.k) break;
+                    const float sc = c == 0 ? sum[t][0] : c == 1 ? sum[t][1] : c == 2 ? sum[t][2] : sum[t][3];
+                    const float wc = c == 0 ? wv[t][0] : c == 1 ? wv[t][1] : c == 2 ? wv[t][2] : wv[t][3];
+                    const float v = __fdiv_rn(sc, P.nf);                                      // line 10: one division by n
+                    P.out_idx[r] = int32_t(pc[t] + c);
+                    P.out_val[r] = v;
+                    if (ONE)
+                        for (int q = 0; q < peers.n; ++q) peers.dst[q][r] = v;        // Eq. 3's values, sent as they are made
+                    ++r;
+                    if (weights) weights[pc[t] + c] = __fsub_rn(wc, __fmul_rn(P.lr, v));      // line 12
+                }
             }
     }
     if (ONE && peers.tag != 0u) {
