@@ -54,6 +54,7 @@ constexpr uint32_t NCOARSE = 1u << 13;
 constexpr int FINE_SHIFT = 9;                                  // key >> 9: 22-bit fine prefix
 constexpr uint32_t WIN = 64;                                   // coarse bins covered above b_lo
 constexpr uint32_t NFINE = WIN * 512;
+constexpr uint32_t LOCAL_CB = NCOARSE / 512;                   // coarse bins above the bound whose fine bins a block counts in shared memory
 constexpr uint32_t DH_BINS = 2048;                             // digit histogram of one radix pass
 constexpr uint32_t DH_PASSES = 8;
 constexpr uint32_t SAMPLE_GRANULE = 128;                       // coordinates one warp samples at a time
@@ -318,6 +319,7 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
         // ---------------- P2: filter pass ----------------------------------------------------------
         clear_outputs();                                               // hidden behind the stream
         for (uint32_t i = tid; i <= WIN; i += TK_THREADS) s.cw[i] = 0;
+        for (uint32_t i = tid; i < LOCAL_CB * 512u; i += TK_THREADS) s.hist[i] = 0;
         if (tid == 0) s.mcount = 0;
         __syncthreads();
         seg_cnt = 0;
@@ -334,7 +336,10 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
                 const uint32_t key = ring[(done + lane) & 63u];
                 const uint32_t cb = (key >> COARSE_SHIFT) - b_lo;
                 atomicAdd(&s.cw[cb < WIN ? cb : WIN], 1u);
-                if (cb < WIN) atomicAdd(&P.fine_hist[(key >> FINE_SHIFT) - fine_base], 1u);
+                // the 22-bit prefixes just above the bound -- where error feedback piles the coordinates up, a few hot bins
+                // late in a run -- are counted per block in shared memory and added to the global histogram once
+                if (cb < LOCAL_CB) atomicAdd(&s.hist[(key >> FINE_SHIFT) - fine_base], 1u);
+                else if (cb < WIN) atomicAdd(&P.fine_hist[(key >> FINE_SHIFT) - fine_base], 1u);
             }
             done += cnt;
             __syncwarp();
@@ -420,6 +425,10 @@ __global__ void __launch_bounds__(TK_THREADS, TK_BLOCKS_PER_SM) topk_select_kern
         for (uint32_t i = tid; i <= WIN; i += TK_THREADS) {
             const uint32_t h = s.cw[i];
             if (h) atomicAdd(&P.coarse_win[i], h);
+        }
+        for (uint32_t i = tid; i < LOCAL_CB * 512u; i += TK_THREADS) {
+            const uint32_t h = s.hist[i];
+            if (h) atomicAdd(&P.fine_hist[i], h);
         }
         if (tid == 0 && s.mcount) atomicAdd(&P.ctrl[CT_CAND], s.mcount);
         SC_STAMP(4);
