@@ -31,7 +31,7 @@ MAX_BATCHES = 24                     # distinct gradient batches kept resident; 
 
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this
 # command with --batches 2) by workload and kernel, with the day of the capture; absent: not captured.
-NCU_TRAFFIC = {"resnet50": {"learner_pass_kernel": 2.4326e9, "topk_select_kernel": 2.205e8, "captured": "2026-11-25"},
+NCU_TRAFFIC = {"resnet50": {"learner_pass_kernel": 2.4326e9, "topk_select_kernel": 2.119e8, "captured": "2026-11-25"},
                "resnet50_n16": {"learner_pass_kernel": 4.8896e9, "captured": "2026-11-25"}}
 
 
